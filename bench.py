@@ -1,0 +1,371 @@
+#!/usr/bin/env python
+"""Benchmark of the HeatKV hot path on B200.
+
+One "step" = one whole generation sweep of the 2B-class single-layer workload (16 heads,
+d=128, 13 scales = 10 521 tokens, batch 2 = one cond/uncond image pair, 20x KV compression):
+for every scale, the eviction before the scale, the ragged attention over the retained keys
+plus the scale's own keys, and the append/compaction of the new K/V.  The schedule comes
+from the library's own calibration kernel run once on seeded samples before timing (the
+paper computes it offline, once per model and budget).
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference]
+
+Prints ONE JSON line (rank 0).  With N > 1 (torchrun) every rank runs an independent replica
+of the workload on its own GPU -- the path has no exchange step -- and the value is the sum of
+images over the slowest rank's time.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import math
+import os
+import subprocess
+import sys
+import threading
+import time
+
+import numpy as np
+import torch
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+sys.path.insert(0, ROOT)
+
+import heatkv_workloads as W  # noqa: E402
+
+B_BUDGET = 1.0 / 20.0
+CALIB_SEEDS = (100, 101, 102, 103)
+DATA_SEED = 0
+METRIC = "images_per_sec_scale_step_attention_2b_single_layer_20x"
+UNIT = "images/s"
+
+
+def peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        p = json.load(open(path))
+        return {"hbm_gbs": p["hbm_gbs"], "bf16_tflops": p["bf16_tflops"],
+                "bf16_tflops_sustained": p.get("bf16_tflops_sustained", p["bf16_tflops"]), "source": "measured"}
+    return {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0, "source": "fallback"}
+
+
+class ClockSampler:
+    """Samples SM clocks and throttle reasons with nvidia-smi while the timed region runs."""
+    Q = ("clocks.sm,clocks.max.sm,clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
+         "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, index: int):
+        self.index, self.proc, self.lines = index, None, []
+
+    def start(self):
+        try:
+            self.proc = subprocess.Popen(["nvidia-smi", f"--id={self.index}", f"--query-gpu={self.Q}",
+                                          "--format=csv,noheader,nounits", "-lms", "100"],
+                                         stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+            self.thread = threading.Thread(target=self._read, daemon=True)
+            self.thread.start()
+        except Exception:
+            self.proc = None
+
+    def _read(self):
+        for line in self.proc.stdout:
+            self.lines.append(line.strip())
+
+    def stop(self):
+        if self.proc is None:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
+        self.proc.terminate()
+        try:
+            self.proc.wait(timeout=5)
+        except Exception:
+            self.proc.kill()
+        sm, mx, reasons = [], [], set()
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        for line in self.lines:
+            parts = [x.strip() for x in line.split(",")]
+            if len(parts) < 6:
+                continue
+            try:
+                sm.append(float(parts[0]))
+                mx.append(float(parts[1]))
+            except ValueError:
+                continue
+            for n, v in zip(names, parts[2:6]):
+                if v.lower().startswith("active"):
+                    reasons.add(n)
+        return {"sm_mhz": float(np.median(sm)) if sm else None, "sm_max_mhz": max(mx) if mx else None,
+                "reasons": sorted(reasons), "samples": len(sm)}
+
+
+def attention_flops(shape, am, n_seq):
+    """Algorithmic flops of every (step) attention launch: 4*d*t_k*n_vis summed over (seq, head),
+    n_vis = retained prior keys + the scale's own keys."""
+    t = shape.t
+    out = []
+    for k in range(shape.K):
+        tot = 0
+        for l in range(shape.L):
+            for h in range(shape.H):
+                prior = sum(t[i] for i in range(k) if (int(am[k, l, h]) >> i) & 1)
+                tot += 4 * shape.d * t[k] * (prior + t[k])
+        out.append(tot * n_seq)
+    return out
+
+
+def oracle_unit_seconds(shape, n_units, bias):
+    """Times the CPU oracle (attention of all 13 steps + cache contents) on `n_units`
+    (seq, head) pairs of the workload.  Returns (seconds, threads)."""
+    from oracle import heatkv_oracle as O
+    scores = W.synthetic_scas(shape, 0)
+    sch = O.heatkv_schedule(scores, B_BUDGET, shape.s, shape.sides)
+    q, k, v = W.qkv_layer(shape, DATA_SEED, 0, n_seq=1)
+    f = lambda x: O.bf16_bits_to_f64(W.bf16_bits(x))
+    qh, kh, vh = f(q), f(k), f(v)
+    kb, vb = W.bf16_bits(k), W.bf16_bits(v)
+    sm = 1.0 / math.sqrt(shape.d)
+    t0 = time.perf_counter()
+    for u in range(n_units):
+        h = u % shape.H
+        for step in range(1, shape.K + 1):
+            lo, hi = (shape.c[step - 2] if step > 1 else 0), shape.c[step - 1]
+            brow = bias[0, step - 1, h].astype(np.float64)
+            O.scale_attention(qh[0, h, lo:hi], kh[0, h], vh[0, h], sch, step, 0, h, sm, brow)
+            if step < shape.K:
+                O.cache_after_layer(kb[0, h], vb[0, h], sch, step, 0, h)
+    dt = time.perf_counter() - t0
+    return dt, torch.get_num_threads()
+
+
+def run_reference(args, rank):
+    """Reference arm: the CPU oracle as it stands, timed on the host cores."""
+    if rank != 0:
+        return
+    shape = W.CFG2
+    bias = W.seg_bias_current_scale(shape, DATA_SEED)
+    units_per_step = 4
+    for _ in range(args.warmup):
+        oracle_unit_seconds(shape, 1, bias)
+    total = 0.0
+    threads = 1
+    for _ in range(args.steps):
+        dt, threads = oracle_unit_seconds(shape, units_per_step, bias)
+        total += dt
+    units_per_image = shape.n_seq * shape.H
+    sec_per_image = total / (args.steps * units_per_step) * units_per_image
+    value = 1.0 / sec_per_image
+    sample = f"{units_per_step} of {units_per_image} (seq, head) units per step, all 13 scales, extrapolated"
+    line = {"impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus,
+            "steps": args.steps, "warmup": args.warmup, "ms_per_step": 1e3 * sec_per_image,
+            "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+            "config": {"workload": W.CFG2.name, "budget": B_BUDGET, "n_seq": shape.n_seq},
+            "cpu_baseline": {"value": value, "unit": UNIT, "cores": threads, "kind": "oracle", "sample": sample},
+            "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+            "gpu_launches": 0}
+    print(json.dumps(line), flush=True)
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=20)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--layout", default="paged", choices=["paged", "ragged"])
+    ap.add_argument("--kernel", default="auto", choices=["auto", "generic", "tcgen05"])
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    args = ap.parse_args()
+    args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
+
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    if args.impl == "reference":
+        run_reference(args, rank)
+        return
+
+    import paper_2605_14877_b200 as hk
+    from paper_2605_14877_b200.sweep import Session
+
+    torch.cuda.set_device(local)
+    dev = torch.device("cuda", local)
+    dist = None
+    if world > 1:
+        import torch.distributed as dist_
+        dist = dist_
+        dist.init_process_group("nccl", device_id=dev)
+
+    shape = W.CFG2
+    layout = hk.LAYOUT_PAGED if args.layout == "paged" else hk.LAYOUT_RAGGED
+    kernel = {"auto": hk.KERNEL_AUTO, "generic": hk.KERNEL_GENERIC, "tcgen05": hk.KERNEL_TCGEN05}[args.kernel]
+    n_seq = shape.n_seq
+    ses = Session(shape.L, shape.H, shape.d, shape.t, shape.s,
+                  pool_rows=n_seq * shape.L * shape.H * (shape.c[-2] + 64 * shape.K), layout=layout,
+                  kernel=kernel, device=str(dev))
+    bias_np = W.seg_bias_current_scale(shape, DATA_SEED)
+    bias = torch.from_numpy(bias_np).to(dev)
+
+    # ---- offline part (untimed): calibration on seeded samples -> S-CAS -> static schedule
+    beta = torch.zeros(shape.L, shape.H, shape.K, shape.K, dtype=torch.float32, device=dev)
+    ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    calib_ms = 0.0
+    for seed in CALIB_SEEDS:
+        q, k, v = W.qkv_layer(shape, seed, 0, device=dev)
+        ev0.record()
+        for step in range(shape.K):
+            lo, hi = ses.step_slices(step)
+            qs, ks = q[:, :, lo:hi], k[:, :, :hi]
+            hk.heatkv_calibrate_scores(ses.ctx, 0, step, n_seq, qs, ks, None, hk.Strides.of(qs, ks), bias[0, step],
+                                       beta, None)
+        ev1.record()
+        torch.cuda.synchronize()
+        calib_ms += ev0.elapsed_time(ev1)
+        del q, k, v
+    _, scas, _ = hk.heatkv_finalize_scores(ses.ctx, beta, len(CALIB_SEEDS) * n_seq, shape.L, shape.H, shape.K)
+    sch = ses.schedule(scas=scas, b=B_BUDGET)
+    am, km, nk, budget = hk.heatkv_schedule_masks(sch, shape.K, shape.L, shape.H)
+    flops = attention_flops(shape, am, n_seq)
+    calib_flops = sum(2 * shape.d * shape.t[k] * shape.c[k] for k in range(shape.K)) * shape.H * n_seq * len(CALIB_SEEDS)
+
+    # ---- device-resident inputs of the timed workload
+    q, k, v = W.qkv_layer(shape, DATA_SEED, 0, device=dev)
+    out = torch.zeros_like(q)
+    flush = torch.empty(256 << 20, dtype=torch.uint8, device=dev)
+    stream = torch.cuda.current_stream()
+
+    def sweep(events=None):
+        ids = [hk.heatkv_seq_open(ses.ctx, sch) for _ in range(n_seq)]
+        for step in range(shape.K):
+            ses.pre_step(ids, step)
+            lo, hi = ses.step_slices(step)
+            qs, ks, vs, os_ = q[:, :, lo:hi], k[:, :, lo:hi], v[:, :, lo:hi], out[:, :, lo:hi]
+            st = hk.Strides.of(qs, ks, os_)
+            if events is not None:
+                events[step][0].record(stream)
+            hk.heatkv_scale_attention(ses.ctx, ids, 0, step, qs, ks, vs, st, bias[0, step], os_)
+            if events is not None:
+                events[step][1].record(stream)
+            hk.heatkv_append_compact(ses.ctx, ids, 0, step, ks, vs, st)
+        for i in ids:
+            hk.heatkv_seq_close(ses.ctx, i)
+
+    def barrier():
+        torch.cuda.synchronize()
+        if dist is not None:
+            dist.barrier()
+            torch.cuda.synchronize()
+
+    for _ in range(args.warmup):
+        sweep()
+    barrier()
+
+    sampler = ClockSampler(local)
+    sampler.start()
+    launches0 = hk.heatkv_launch_count(ses.ctx)
+    step_events = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True))
+                   for _ in range(args.steps)]
+    kern_events = [[(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True))
+                    for _ in range(shape.K)] for _ in range(args.steps)]
+    barrier()
+    for it in range(args.steps):
+        flush.fill_(it & 0xff)                         # evict L2 between timed steps (untimed)
+        step_events[it][0].record(stream)
+        sweep(kern_events[it])
+        step_events[it][1].record(stream)
+    barrier()
+    launches = hk.heatkv_launch_count(ses.ctx) - launches0
+    total_ms = sum(a.elapsed_time(b) for a, b in step_events)
+    per_step_ms = [[a.elapsed_time(b) for a, b in ke] for ke in kern_events]
+    clocks = sampler.stop()
+    assert hk.heatkv_device_status(ses.ctx) == 0
+
+    # ---- end to end: host (pinned) inputs, copies inside the timed region
+    hq, hk_, hv = (x.cpu().pin_memory() for x in (q, k, v))
+    hout = torch.empty_like(hq).pin_memory()
+    dq, dk, dv, dout = (torch.empty_like(q) for _ in range(4))
+    e2e_steps = max(3, min(args.steps, 5))
+
+    def sweep_e2e():
+        ids = [hk.heatkv_seq_open(ses.ctx, sch) for _ in range(n_seq)]
+        for step in range(shape.K):
+            lo, hi = ses.step_slices(step)
+            for src, dst in ((hq, dq), (hk_, dk), (hv, dv)):
+                dst[:, :, lo:hi].copy_(src[:, :, lo:hi], non_blocking=True)
+            ses.pre_step(ids, step)
+            ses.run_layer_step(ids, 0, step, dq, dk, dv, dout, bias[0, step])
+            hout[:, :, lo:hi].copy_(dout[:, :, lo:hi], non_blocking=True)
+        for i in ids:
+            hk.heatkv_seq_close(ses.ctx, i)
+
+    sweep_e2e()
+    barrier()
+    t0 = time.perf_counter()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record(stream)
+    for _ in range(e2e_steps):
+        sweep_e2e()
+    e1.record(stream)
+    barrier()
+    e2e_ms = max(e0.elapsed_time(e1), 1e3 * (time.perf_counter() - t0)) / e2e_steps
+    h2d = 3 * q.numel() * 2
+    d2h = q.numel() * 2
+
+    # ---- aggregate over ranks (replicas): slowest rank's time
+    if dist is not None:
+        tt = torch.tensor([total_ms, e2e_ms], device=dev)
+        dist.all_reduce(tt, op=dist.ReduceOp.MAX)
+        total_ms, e2e_ms = (float(x) for x in tt.cpu())
+    images_per_step = 1 * world                     # one cond/uncond pair per replica
+    ms_per_step = total_ms / args.steps
+    value = images_per_step / (ms_per_step * 1e-3)
+
+    # ---- roofline of the dominant kernel: the attention launches of the large steps
+    pk = peaks()
+    attn_ms = np.array(per_step_ms).mean(axis=0)                  # [K] mean duration per launch
+    big = [kk for kk in range(shape.K) if shape.t[kk] >= 1024]
+    dom_flops = sum(flops[kk] for kk in big)
+    dom_ms = float(sum(attn_ms[kk] for kk in big))
+    achieved = dom_flops / (dom_ms * 1e-3) / 1e12
+    uncompressed_kv_bytes = sum(2 * shape.c[kk] * shape.d * 2 for kk in range(shape.K)) * shape.H * n_seq
+    line = {
+        "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
+        "warmup": args.warmup, "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak",
+        "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
+        "config": {"workload": shape.name, "L": shape.L, "H": shape.H, "d": shape.d, "scales": shape.K,
+                   "tokens": shape.n_tokens, "n_seq": n_seq, "budget": B_BUDGET, "policy": "heatkv", "s": shape.s,
+                   "layout": args.layout, "kernel": args.kernel, "l2": "256 MB flush write between timed steps",
+                   "one_image": "cond/uncond pair through one layer; x32 layers for a 2B-class model",
+                   "n_k": [int(x) for x in nk], "replicas": world},
+        "effective_kv_tb_per_s": uncompressed_kv_bytes / (float(attn_ms.sum()) * 1e-3) / 1e12,
+        "attention_ms_per_scale": [round(float(x), 5) for x in attn_ms],
+        "attention_tflops_all_scales": sum(flops) / (float(attn_ms.sum()) * 1e-3) / 1e12,
+        "images_per_s_32_layers_extrapolated": value / 32.0,
+        "calibration": {"ms_per_sample_batch": calib_ms / len(CALIB_SEEDS),
+                        "tflops": calib_flops / (calib_ms * 1e-3) / 1e12, "samples": len(CALIB_SEEDS) * n_seq},
+        "roofline": {"bound": "tensor", "kernel": "scale attention, scales with t_k >= 1024 (4 launches per step)",
+                     "achieved": achieved, "peak": pk["bf16_tflops"], "unit": "TFLOP/s",
+                     "frac": achieved / pk["bf16_tflops"], "peak_source": pk["source"] + " burst bf16",
+                     "traffic": None},
+        "e2e": {"value": images_per_step / (e2e_ms * 1e-3), "unit": UNIT, "h2d_bytes_per_step": h2d,
+                "d2h_bytes_per_step": d2h, "steps": e2e_steps},
+        "gpu_launches": int(launches),
+        "clocks": clocks,
+    }
+    if rank == 0 and world == 1 and not args.no_cpu_baseline:
+        bias_cpu = bias_np
+        n_units = 16
+        dt, threads = oracle_unit_seconds(shape, n_units, bias_cpu)
+        sec_per_image = dt / n_units * (shape.n_seq * shape.H)
+        line["cpu_baseline"] = {"value": 1.0 / sec_per_image, "unit": UNIT, "cores": threads, "kind": "oracle",
+                                "sample": f"{n_units} of {shape.n_seq * shape.H} (seq, head) units, all 13 scales "
+                                          f"(attention + cache contents), extrapolated; {dt:.1f} s of CPU work"}
+    hk.heatkv_schedule_free(sch)
+    ses.close()
+    if dist is not None:
+        dist.barrier()
+        dist.destroy_process_group()
+    if rank == 0:
+        print(json.dumps(line), flush=True)
+
+
+if __name__ == "__main__":
+    main()

@@ -1,0 +1,220 @@
+/*
+ * heatkv.h -- C ABI of the B200 (sm_100a) HeatKV hot path.
+ *
+ * HeatKV (head-tuned KV-cache compression for visual autoregressive, next-scale
+ * models) prunes the KV cache per attention head and per source scale with a static
+ * schedule derived from calibrated attention statistics.  This library holds the
+ * data-parallel part: the calibration reduction (Sec. 3.1), the schedule builder
+ * (Sec. 3.2, 3.3, Appendix A), the per-head cache with append / eviction, and the
+ * per-scale-step attention over the retained keys.
+ *
+ * Conventions
+ *  - Scales ("steps"), layers and heads are 0-based here: step = k-1 for the paper's
+ *    scale k, so t[step] tokens are generated at `step` and c[step] = t[0]+..+t[step].
+ *  - Activations are bf16, shaped [n_seq, H, t_step, d] with d contiguous; the other
+ *    three strides are given in elements by heatkv_strides (NULL = densely packed).
+ *    Base pointers must be 16-byte aligned and strides multiples of 8 elements.
+ *  - Every pointer is marked HOST or DEVICE.  Device buffers belong to the caller (the
+ *    library never allocates or frees device memory); the library owns only the host
+ *    objects behind heatkv_ctx / heatkv_schedule.  Kernels are enqueued on the given
+ *    CUDA stream (a cudaStream_t passed as void*, NULL = default stream) and calls return
+ *    without waiting, except the calls documented as synchronising.
+ *  - Every function returns HEATKV_OK (0) or a negative heatkv_status.  Nothing throws or
+ *    aborts across this boundary; a call that fails leaves cache and context unchanged.
+ *  - A context is not thread-safe; use one context per thread or lock around it.
+ */
+#ifndef HEATKV_H_
+#define HEATKV_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+#define HEATKV_MAX_K 16          /* at most 16 scales (mask words are 16 bit)        */
+#define HEATKV_MAX_BATCH 128     /* sequences per attention / append call            */
+#define HEATKV_PAGE_TOKENS 64    /* rows per cache page and per key half-tile        */
+
+typedef enum {
+  HEATKV_OK = 0,
+  HEATKV_ERR_INVALID_ARG = -1,
+  HEATKV_ERR_SHAPE_MISMATCH = -2,
+  HEATKV_ERR_BUDGET_INFEASIBLE = -3,   /* b*c_{K-1} < c_s, or the removal list ran out */
+  HEATKV_ERR_OUT_OF_PAGES = -4,        /* pool or metadata region exhausted            */
+  HEATKV_ERR_BAD_STEP_ORDER = -5,
+  HEATKV_ERR_NAN_SCORE = -6,
+  HEATKV_ERR_DEVICE_TIMEOUT = -7,      /* a bounded device-side wait gave up           */
+  HEATKV_ERR_CUDA = -8,
+  HEATKV_ERR_HOST_MEMORY = -9
+} heatkv_status;
+
+typedef enum { HEATKV_LAYOUT_RAGGED = 0, HEATKV_LAYOUT_PAGED = 1 } heatkv_layout;
+
+typedef enum {
+  HEATKV_POLICY_HEATKV = 0,   /* Algorithm 1, head-scale units, orders O_i from S-CAS      */
+  HEATKV_POLICY_BINARY = 1,   /* Algorithm 1, head units, one order O from CAS            */
+  HEATKV_POLICY_NAIVE = 2,    /* Sec. 3.3 boundary policy: prune before a scale, not after */
+  HEATKV_POLICY_EXPLICIT = 3  /* per-head token fraction (no counterpart in the paper)     */
+} heatkv_policy;
+
+typedef enum {
+  HEATKV_ACCOUNT_PHYSICAL = 0, /* layers not yet run hold what they held at scale start   */
+  HEATKV_ACCOUNT_LITERAL = 1   /* Algorithm 2 exactly as printed                          */
+} heatkv_accounting;
+
+typedef enum {
+  HEATKV_KERNEL_AUTO = 0,      /* tensor-memory kernel for large steps, generic otherwise */
+  HEATKV_KERNEL_GENERIC = 1,   /* warp-level MMA kernel for every step                    */
+  HEATKV_KERNEL_TCGEN05 = 2    /* tcgen05 / TMEM / TMA kernel wherever its shape rules allow */
+} heatkv_kernel_choice;
+
+typedef struct heatkv_ctx heatkv_ctx;
+typedef struct heatkv_schedule heatkv_schedule;
+
+typedef struct {
+  int32_t L, H, d, K;            /* layers, heads per layer, head dim (64 or 128), scales  */
+  int32_t t[HEATKV_MAX_K];       /* tokens per scale, t_k = w_k * h_k (Sec. 3.1)           */
+  int32_t s;                     /* sink scales always kept (Sec. 3.2); 0 allowed          */
+  int32_t layout;                /* heatkv_layout                                           */
+  int32_t kernel;                /* heatkv_kernel_choice                                    */
+  float sm_scale;                /* logit scale; <= 0 selects 1/sqrt(d)                    */
+  void* arena;                   /* DEVICE, caller-owned, 1024-byte aligned                */
+  uint64_t arena_bytes;          /* metadata region + K pool + V pool                      */
+  uint64_t meta_bytes;           /* bytes of the arena set aside for plans; 0 = default    */
+} heatkv_config;
+
+typedef struct {                 /* element strides of the [n_seq, H, t, d] activations    */
+  int64_t q_seq, q_head, q_tok;
+  int64_t kv_seq, kv_head, kv_tok;   /* shared by k and v                                  */
+  int64_t o_seq, o_head, o_tok;
+} heatkv_strides;
+
+typedef struct {
+  uint64_t pool_rows;            /* rows (tokens) the K pool and the V pool can hold        */
+  uint64_t reserved_rows;        /* rows reserved by open sequences                         */
+  uint64_t used_tokens;          /* tokens held right now by open sequences                 */
+  uint64_t peak_reserved_rows;   /* high-water mark of reserved_rows                        */
+  uint64_t meta_bytes_used;
+  uint32_t open_seqs;
+  uint32_t plans;                /* schedules whose plan is resident                        */
+} heatkv_alloc_stats;
+
+/* Context: validates the shape, splits the arena into a metadata region and the K / V
+ * pools, zero-fills the pools (enqueued on `stream`).  The arena must outlive the context. */
+int heatkv_create(const heatkv_config* cfg /*HOST*/, void* stream, heatkv_ctx** out /*HOST*/);
+int heatkv_destroy(heatkv_ctx* ctx);
+
+/* Sec. 3.1, Eq. 2 -- scale attention mass.  For one (layer, step) and n_seq calibration
+ * sequences: attention of the t[step] queries over ALL c[step] keys (no pruning), fused
+ * with the per-row probability mass on each source scale; the mean over rows is added to
+ * beta_accum[layer][h][step][0..step] for every head (sum over the n_seq sequences; every
+ * sequence counts as one data point d).  The attention matrix is never written out.
+ *   q       DEVICE bf16 [n_seq,H,t[step],d]   strides q_*
+ *   k_full  DEVICE bf16 [n_seq,H,c[step],d]   strides kv_*  (all scales up to `step`)
+ *   v_full  DEVICE bf16 like k_full, or NULL when `out` is NULL
+ *   seg_bias DEVICE fp32 [H][K] additive logit bias per source scale, or NULL
+ *   beta_accum DEVICE fp32 [L][H][K][K], zero-initialised by the caller before the first call
+ *   out     DEVICE bf16 [n_seq,H,t[step],d] strides o_*: the attention output, or NULL    */
+int heatkv_calibrate_scores(heatkv_ctx* ctx, int layer, int step, int n_seq, const void* q,
+                            const void* k_full, const void* v_full, const heatkv_strides* st,
+                            const float* seg_bias, float* beta_accum, void* out, void* stream);
+
+/* Text after Eq. 2, Eq. 3 and Eq. 4 -- copies beta_accum to the host (synchronises
+ * `stream`), divides by n_samples = |D| and reduces in fp64:
+ *   beta HOST [L][H][K][K], scas HOST [L][H][K] (0 outside s < k < K), cas HOST [L][H].
+ * Any of the three outputs may be NULL.  HEATKV_ERR_NAN_SCORE if a value is not finite. */
+int heatkv_finalize_scores(heatkv_ctx* ctx, const float* beta_accum /*DEVICE*/, int n_samples,
+                           double* beta, double* scas, double* cas, void* stream);
+
+/* Sec. 3.2 (Eq. 5), Sec. 3.3 (Algorithm 1), Appendix A (Algorithm 2) -- pure host code.
+ * Ranks heads per source scale by ascending S-CAS (ties: ascending l*H+h), computes N_k,
+ * the sets G_k, E_k (GreedyEarlyPruning) and A_k = G_{k-1} u E_k for every scale.
+ *   scas HOST [L][H][K]  (HEATKV, NAIVE)      cas HOST [L][H]  (BINARY)
+ *   fraction HOST [L][H] (EXPLICIT: the head stores scales 1..j, the largest prefix with
+ *            c_j <= ceil(fraction * c_{K-1}), at least the sinks, and never evicts)
+ *   b in (0,1]: the budget is B = floor(b * L*H * c_{K-1}) tokens (ignored by EXPLICIT).
+ * Only L, H, K, t, s of cfg are read.                                                    */
+int heatkv_build_schedule(const heatkv_config* cfg, const double* scas, const double* cas,
+                          int policy, int accounting, double b, const double* fraction,
+                          heatkv_schedule** out);
+int heatkv_schedule_free(heatkv_schedule* sch);
+
+/* Schedule as bit masks, HOST arrays of K*L*H uint16 indexed [step][layer][head]:
+ *   attn_mask bit i (i < step): source scale i is in the cache and visible at `step`,
+ *             i.e. i is a sink or (i,l,h) is not in A_step;
+ *   keep_mask bit i (i <= step): source scale i is stored once the layer ran at `step`,
+ *             i.e. i is a sink or (i,l,h) is not in G_step (last step: unchanged, nothing
+ *             is appended because the last scale is never cached).
+ *   n_k HOST [K] (N_k, 0 for the last step), budget_tokens = B (-1 for EXPLICIT).
+ * Any output may be NULL.                                                                */
+int heatkv_schedule_masks(const heatkv_schedule* sch, uint16_t* attn_mask, uint16_t* keep_mask,
+                          int32_t* n_k, int64_t* budget_tokens);
+
+/* Peak number of cached tokens over all checkpoints (scale start and after every layer)
+ * and the pool rows one sequence reserves under `layout`.                                */
+int heatkv_schedule_footprint(const heatkv_schedule* sch, int layout, int64_t* peak_tokens,
+                              int64_t* reserved_rows);
+
+/* The plan a sequence of this schedule runs under `layout`, as the flat int32 table the
+ * kernels read (HOST copy, for inspection and tests): a 20-word header {L, H, K, n_desc,
+ * word offsets of: desc, attn_begin, attn_cnt, app_begin, app_cnt, order, move, pre_begin,
+ * pre_cnt, post_begin, post_cnt, then n_move, total_words, 3 spare} followed by the tables.
+ * desc = {row relative to the reservation, n_valid | source_scale << 8}; move = {src, dst, n, 0};
+ * the per-(step, layer, head) tables are indexed (step*L + layer)*H + head.
+ * Call with words == NULL to get *n_words, then with a buffer of that many int32.        */
+int heatkv_schedule_plan(const heatkv_schedule* sch, int layout, int32_t* words, int64_t* n_words);
+
+/* Admit / retire one image.  Opening reserves the sequence's rows for its whole life (the
+ * schedule is static, so the reservation and every page table are known up front) and, on
+ * first use of a schedule, uploads its plan on `stream`.  HEATKV_ERR_OUT_OF_PAGES if the
+ * pool or the metadata region cannot hold it.                                            */
+int heatkv_seq_open(heatkv_ctx* ctx, const heatkv_schedule* sch, void* stream, int* seq_id);
+int heatkv_seq_close(heatkv_ctx* ctx, int seq_id);
+
+/* Sec. 3.3 -- cache update for one layer.
+ *   k_new != NULL: after layer `layer` ran at `step`: store the step's K/V for every head
+ *     whose (step,l,h) is not in G_step and drop the head-scales of G_step \ A_step of this
+ *     layer ("evicted immediately after their layer has executed").  The last step stores
+ *     nothing.  k_new, v_new DEVICE bf16 [n_seq,H,t[step],d], strides kv_*.
+ *   k_new == NULL: before `step` starts: drop the head-scales of E_step ("evicted before
+ *     scale k starts") in `layer`, or in all layers when layer < 0.
+ * Survivors keep their order.  In the paged layout eviction moves no data.               */
+int heatkv_append_compact(heatkv_ctx* ctx, const int* seq_ids /*HOST*/, int n_seq, int layer,
+                          int step, const void* k_new, const void* v_new,
+                          const heatkv_strides* st, void* stream);
+
+/* Attention of one layer at one step (Sec. 3.1 notation; Sec. 3.3 for the visible set):
+ * out = softmax(sm_scale * q K^T + bias) V over the retained prior head-scales (ascending
+ * scale, raster order inside) followed by the step's own t[step] keys, which always come
+ * from k_new / v_new and are all visible.  bf16 operands, fp32 accumulation, probabilities
+ * rounded to bf16 before the PV product.
+ *   q, k_new, v_new DEVICE bf16 [n_seq,H,t[step],d]; seg_bias DEVICE fp32 [H][K] or NULL;
+ *   out DEVICE bf16 [n_seq,H,t[step],d].                                                 */
+int heatkv_scale_attention(heatkv_ctx* ctx, const int* seq_ids /*HOST*/, int n_seq, int layer,
+                           int step, const void* q, const void* k_new, const void* v_new,
+                           const heatkv_strides* st, const float* seg_bias, void* out,
+                           void* stream);
+
+/* Introspection (host state only unless noted). */
+int heatkv_cache_bytes(heatkv_ctx* ctx, int seq_id, uint64_t* actual, uint64_t* reserved);
+/* Global token indices c_{i-1}+j of the tokens head (layer, head) holds now; idx HOST with
+ * room for c_{K-1} entries. */
+int heatkv_retained_indices(heatkv_ctx* ctx, int seq_id, int layer, int head, int32_t* idx, int* n);
+/* Gathers the head's cached K and V rows in logical order into DEVICE buffers of
+ * n*d bf16 each (enqueued on `stream`). */
+int heatkv_export_head(heatkv_ctx* ctx, int seq_id, int layer, int head, void* k_out, void* v_out,
+                       void* stream);
+int heatkv_allocator_stats(heatkv_ctx* ctx, heatkv_alloc_stats* out);
+/* Kernels launched by this context so far. */
+int heatkv_launch_count(heatkv_ctx* ctx, uint64_t* n);
+/* Reads the device-side status word (synchronises `stream`): HEATKV_OK or
+ * HEATKV_ERR_DEVICE_TIMEOUT if a bounded wait inside a kernel ran out. */
+int heatkv_device_status(heatkv_ctx* ctx, void* stream);
+const char* heatkv_strerror(int status);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* HEATKV_H_ */

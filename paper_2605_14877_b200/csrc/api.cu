@@ -1,0 +1,694 @@
+// C ABI of libheatkv: context, arena bookkeeping, sequence admission and the launch logic
+// of every entry point declared in heatkv.h.
+#include <cmath>
+#include <cstring>
+#include <map>
+#include <memory>
+#include <new>
+#include <vector>
+
+#include "device_common.cuh"
+#include "internal.h"
+
+namespace heatkv {
+cudaError_t launch_attn_generic(const AttnParams& p, int d, int n_seq, bool calib, cudaStream_t stream);
+cudaError_t launch_append(const CopyParams& p, int n_seq, cudaStream_t stream);
+cudaError_t launch_compact(const CopyParams& p, int n_seq, cudaStream_t stream);
+struct TcState;
+int tc_create(const heatkv_config& cfg, void* k_pool, void* v_pool, uint64_t pool_rows, TcState** out);
+void tc_destroy(TcState* st);
+bool tc_supported(const TcState* st, const AttnParams& p, int d, int n_seq, bool calib);
+cudaError_t launch_attn_tc(TcState* st, const AttnParams& p, int d, int n_seq, bool calib, cudaStream_t stream,
+                           int* launches);
+}  // namespace heatkv
+
+using namespace heatkv;
+
+struct heatkv_schedule {
+  Schedule s;
+};
+
+namespace {
+
+constexpr uint64_t META_ALIGN = 256;
+constexpr uint64_t STATUS_BYTES = 256;
+
+// first-fit allocator over [0, size) in abstract units
+struct RangeAlloc {
+  std::map<uint64_t, uint64_t> free_;   // start -> length
+  void reset(uint64_t start, uint64_t len) {
+    free_.clear();
+    if (len) free_[start] = len;
+  }
+  bool alloc(uint64_t len, uint64_t* start) {
+    for (auto it = free_.begin(); it != free_.end(); ++it) {
+      if (it->second >= len) {
+        *start = it->first;
+        uint64_t rest = it->second - len, s2 = it->first + len;
+        free_.erase(it);
+        if (rest) free_[s2] = rest;
+        return true;
+      }
+    }
+    return false;
+  }
+  void release(uint64_t start, uint64_t len) {
+    auto it = free_.emplace(start, len).first;
+    auto nx = std::next(it);
+    if (nx != free_.end() && it->first + it->second == nx->first) {
+      it->second += nx->second;
+      free_.erase(nx);
+    }
+    if (it != free_.begin()) {
+      auto pv = std::prev(it);
+      if (pv->first + pv->second == it->first) {
+        pv->second += it->second;
+        free_.erase(it);
+      }
+    }
+  }
+};
+
+struct PlanEntry {
+  uint64_t uid = 0;
+  Schedule sched;
+  Plan plan;
+  uint64_t meta_off = 0, meta_len = 0;
+  int refs = 0;
+};
+
+struct Seq {
+  bool open = false;
+  int plan = -1;
+  uint64_t base_row = 0, rows = 0;
+  std::vector<int16_t> done_step;   // per layer: last step whose post-layer update ran (-1 = none)
+  std::vector<int16_t> pre_step;    // per layer: last step whose pre-step eviction ran
+};
+
+inline bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15) == 0; }
+
+}  // namespace
+
+struct heatkv_ctx {
+  heatkv_config cfg;
+  int c[HEATKV_MAX_K];
+  float sm_scale;
+  unsigned char* meta = nullptr;
+  __nv_bfloat16* k_pool = nullptr;
+  __nv_bfloat16* v_pool = nullptr;
+  uint64_t pool_rows = 0, meta_bytes = 0;
+  uint32_t* status = nullptr;
+  RangeAlloc rows, metas;
+  std::vector<std::unique_ptr<PlanEntry>> plans;
+  std::vector<Seq> seqs;
+  uint64_t reserved_rows = 0, peak_reserved = 0, meta_used = 0;
+  uint64_t launches = 0;
+  TcState* tc = nullptr;
+};
+
+namespace {
+
+int find_or_load_plan(heatkv_ctx* ctx, const Schedule& s, cudaStream_t stream, int* idx) {
+  for (size_t i = 0; i < ctx->plans.size(); ++i)
+    if (ctx->plans[i] && ctx->plans[i]->uid == s.uid) { *idx = (int)i; return HEATKV_OK; }
+  if (s.L != ctx->cfg.L || s.H != ctx->cfg.H || s.K != ctx->cfg.K || s.s != ctx->cfg.s)
+    return HEATKV_ERR_SHAPE_MISMATCH;
+  for (int i = 0; i < s.K; ++i)
+    if (s.t[i] != ctx->cfg.t[i]) return HEATKV_ERR_SHAPE_MISMATCH;
+  std::unique_ptr<PlanEntry> e(new (std::nothrow) PlanEntry);
+  if (!e) return HEATKV_ERR_HOST_MEMORY;
+  e->uid = s.uid;
+  e->sched = s;
+  int rc = build_plan(s, ctx->cfg.layout, &e->plan);
+  if (rc != HEATKV_OK) return rc;
+  uint64_t bytes = ((uint64_t)e->plan.blob.size() * 4 + META_ALIGN - 1) / META_ALIGN * META_ALIGN;
+  uint64_t off = 0;
+  bool ok = ctx->metas.alloc(bytes, &off);
+  if (!ok) {                                    // drop resident plans nobody uses and retry
+    for (auto& pe : ctx->plans)
+      if (pe && pe->refs == 0) {
+        ctx->metas.release(pe->meta_off, pe->meta_len);
+        ctx->meta_used -= pe->meta_len;
+        pe.reset();
+      }
+    ok = ctx->metas.alloc(bytes, &off);
+  }
+  if (!ok) return HEATKV_ERR_OUT_OF_PAGES;
+  e->meta_off = off;
+  e->meta_len = bytes;
+  if (cudaMemcpyAsync(ctx->meta + off, e->plan.blob.data(), e->plan.blob.size() * 4, cudaMemcpyHostToDevice,
+                      stream) != cudaSuccess) {
+    ctx->metas.release(off, bytes);
+    return HEATKV_ERR_CUDA;
+  }
+  // the blob is pageable host memory: wait so the vector may be touched again safely
+  if (cudaStreamSynchronize(stream) != cudaSuccess) return HEATKV_ERR_CUDA;
+  ctx->meta_used += bytes;
+  size_t slot = ctx->plans.size();
+  for (size_t i = 0; i < ctx->plans.size(); ++i)
+    if (!ctx->plans[i]) { slot = i; break; }
+  if (slot == ctx->plans.size()) ctx->plans.emplace_back();
+  ctx->plans[slot] = std::move(e);
+  *idx = (int)slot;
+  return HEATKV_OK;
+}
+
+inline Seq* get_seq(heatkv_ctx* ctx, int id) {
+  if (id < 0 || id >= (int)ctx->seqs.size() || !ctx->seqs[id].open) return nullptr;
+  return &ctx->seqs[id];
+}
+
+// scales head (l,h) of the sequence holds right now
+uint16_t stored_mask(const heatkv_ctx* ctx, const Seq& q, int l, int h) {
+  const Schedule& s = ctx->plans[q.plan]->sched;
+  int done = q.done_step[l];
+  uint16_t m = done >= 0 ? s.keep_mask[s.at(done, l, h)] : 0;
+  if (q.pre_step[l] > done && q.pre_step[l] < s.K) m &= s.attn_mask[s.at(q.pre_step[l], l, h)];
+  return m;
+}
+
+// does the eviction before `step` remove anything from layer l?
+bool pre_needed(const Schedule& s, int step, int l) {
+  if (step == 0) return false;
+  for (int h = 0; h < s.H; ++h)
+    if (s.keep_mask[s.at(step - 1, l, h)] & ~s.attn_mask[s.at(step, l, h)]) return true;
+  return false;
+}
+
+int check_strides(const heatkv_ctx* ctx, const heatkv_strides* st, int t, heatkv_strides* out) {
+  const int64_t d = ctx->cfg.d, H = ctx->cfg.H;
+  if (!st) {
+    out->q_tok = out->kv_tok = out->o_tok = d;
+    out->q_head = out->kv_head = out->o_head = d * t;
+    out->q_seq = out->kv_seq = out->o_seq = d * t * H;
+    return HEATKV_OK;
+  }
+  *out = *st;
+  const int64_t* v = &out->q_seq;
+  for (int i = 0; i < 9; ++i)
+    if (v[i] < 0 || (v[i] & 7)) return HEATKV_ERR_INVALID_ARG;
+  if (out->q_tok < d || out->kv_tok < d || out->o_tok < d) return HEATKV_ERR_INVALID_ARG;
+  return HEATKV_OK;
+}
+
+void fill_common(const heatkv_ctx* ctx, AttnParams* p, const heatkv_strides& s) {
+  p->q_seq = s.q_seq; p->q_head = s.q_head; p->q_tok = s.q_tok;
+  p->kv_seq = s.kv_seq; p->kv_head = s.kv_head; p->kv_tok = s.kv_tok;
+  p->o_seq = s.o_seq; p->o_head = s.o_head; p->o_tok = s.o_tok;
+  p->H = ctx->cfg.H; p->K = ctx->cfg.K; p->L = ctx->cfg.L;
+  p->scale_log2 = ctx->sm_scale * 1.4426950408889634f;
+  for (int i = 0; i < HEATKV_MAX_K; ++i) p->c[i] = i < ctx->cfg.K ? ctx->c[i] : 0x7fffffff;
+  p->k_pool = ctx->k_pool; p->v_pool = ctx->v_pool;
+  p->status = ctx->status;
+}
+
+// Validates ids and per-layer progress for a batched call and fills the SeqRef table.
+int gather_seqs(heatkv_ctx* ctx, const int* seq_ids, int n_seq, int layer, int step, SeqRef* refs) {
+  if (!seq_ids || n_seq < 1 || n_seq > HEATKV_MAX_BATCH) return HEATKV_ERR_INVALID_ARG;
+  if (layer < 0 || layer >= ctx->cfg.L || step < 0 || step >= ctx->cfg.K) return HEATKV_ERR_INVALID_ARG;
+  for (int i = 0; i < n_seq; ++i) {
+    Seq* q = get_seq(ctx, seq_ids[i]);
+    if (!q) return HEATKV_ERR_INVALID_ARG;
+    for (int j = 0; j < i; ++j)
+      if (seq_ids[j] == seq_ids[i]) return HEATKV_ERR_INVALID_ARG;
+    const PlanEntry& pe = *ctx->plans[q->plan];
+    if (q->done_step[layer] != step - 1) return HEATKV_ERR_BAD_STEP_ORDER;
+    if (q->pre_step[layer] != step && pre_needed(pe.sched, step, layer)) return HEATKV_ERR_BAD_STEP_ORDER;
+    refs[i].plan = reinterpret_cast<const int32_t*>(ctx->meta + pe.meta_off);
+    refs[i].base_row = (int64_t)q->base_row;
+  }
+  return HEATKV_OK;
+}
+
+}  // namespace
+
+extern "C" {
+
+const char* heatkv_strerror(int status) {
+  switch (status) {
+    case HEATKV_OK: return "ok";
+    case HEATKV_ERR_INVALID_ARG: return "invalid argument";
+    case HEATKV_ERR_SHAPE_MISMATCH: return "shape mismatch between schedule, context or call";
+    case HEATKV_ERR_BUDGET_INFEASIBLE: return "budget infeasible";
+    case HEATKV_ERR_OUT_OF_PAGES: return "cache pool or metadata region exhausted";
+    case HEATKV_ERR_BAD_STEP_ORDER: return "call out of generation order";
+    case HEATKV_ERR_NAN_SCORE: return "score is not finite";
+    case HEATKV_ERR_DEVICE_TIMEOUT: return "a bounded device-side wait ran out";
+    case HEATKV_ERR_CUDA: return "CUDA runtime error";
+    case HEATKV_ERR_HOST_MEMORY: return "host allocation failed";
+    default: return "unknown status";
+  }
+}
+
+int heatkv_create(const heatkv_config* cfg, void* stream_, heatkv_ctx** out) {
+  if (!cfg || !out) return HEATKV_ERR_INVALID_ARG;
+  cudaStream_t stream = static_cast<cudaStream_t>(stream_);
+  if (cfg->L < 1 || cfg->H < 1 || cfg->K < 1 || cfg->K > HEATKV_MAX_K) return HEATKV_ERR_INVALID_ARG;
+  if (cfg->d != 64 && cfg->d != 128) return HEATKV_ERR_INVALID_ARG;
+  if (cfg->s < 0 || cfg->s > (cfg->K > 1 ? cfg->K - 1 : 0)) return HEATKV_ERR_INVALID_ARG;
+  if (cfg->layout != HEATKV_LAYOUT_RAGGED && cfg->layout != HEATKV_LAYOUT_PAGED) return HEATKV_ERR_INVALID_ARG;
+  if (cfg->kernel < HEATKV_KERNEL_AUTO || cfg->kernel > HEATKV_KERNEL_TCGEN05) return HEATKV_ERR_INVALID_ARG;
+  if (!cfg->arena || (reinterpret_cast<uintptr_t>(cfg->arena) & 1023)) return HEATKV_ERR_INVALID_ARG;
+  for (int i = 0; i < cfg->K; ++i)
+    if (cfg->t[i] < 1 || cfg->t[i] > (1 << 20)) return HEATKV_ERR_INVALID_ARG;
+  std::unique_ptr<heatkv_ctx> ctx(new (std::nothrow) heatkv_ctx);
+  if (!ctx) return HEATKV_ERR_HOST_MEMORY;
+  ctx->cfg = *cfg;
+  for (int i = 0, acc = 0; i < cfg->K; ++i) { acc += cfg->t[i]; ctx->c[i] = acc; }
+  ctx->sm_scale = cfg->sm_scale > 0.f ? cfg->sm_scale : 1.0f / std::sqrt((float)cfg->d);
+  uint64_t meta = cfg->meta_bytes;
+  if (meta == 0) meta = std::min<uint64_t>(std::max<uint64_t>(cfg->arena_bytes / 16, 1u << 20), 256u << 20);
+  meta = (meta + 1023) / 1024 * 1024;
+  if (meta < STATUS_BYTES + META_ALIGN || cfg->arena_bytes < meta + 2ull * HEATKV_PAGE_TOKENS * cfg->d * 2)
+    return HEATKV_ERR_INVALID_ARG;
+  const uint64_t row_bytes = (uint64_t)cfg->d * 2;
+  uint64_t rows = (cfg->arena_bytes - meta) / (2 * row_bytes);
+  rows = rows / HEATKV_PAGE_TOKENS * HEATKV_PAGE_TOKENS;
+  if (rows > 0x7fffffffull) rows = 0x7fffffc0ull;
+  ctx->meta = static_cast<unsigned char*>(cfg->arena);
+  ctx->meta_bytes = meta;
+  ctx->k_pool = reinterpret_cast<__nv_bfloat16*>(ctx->meta + meta);
+  ctx->v_pool = ctx->k_pool + rows * cfg->d;
+  ctx->pool_rows = rows;
+  ctx->status = reinterpret_cast<uint32_t*>(ctx->meta);
+  ctx->rows.reset(0, rows);
+  ctx->metas.reset(STATUS_BYTES, meta - STATUS_BYTES);
+  // zero the status word and both pools: half-tiles are read whole, rows past a tile's valid
+  // count must hold finite values
+  if (cudaMemsetAsync(ctx->meta, 0, STATUS_BYTES, stream) != cudaSuccess) return HEATKV_ERR_CUDA;
+  if (cudaMemsetAsync(ctx->k_pool, 0, 2 * rows * row_bytes, stream) != cudaSuccess) return HEATKV_ERR_CUDA;
+  int rc = tc_create(ctx->cfg, ctx->k_pool, ctx->v_pool, rows, &ctx->tc);
+  if (rc != HEATKV_OK) return rc;
+  *out = ctx.release();
+  return HEATKV_OK;
+}
+
+int heatkv_destroy(heatkv_ctx* ctx) {
+  if (!ctx) return HEATKV_ERR_INVALID_ARG;
+  tc_destroy(ctx->tc);
+  delete ctx;
+  return HEATKV_OK;
+}
+
+int heatkv_build_schedule(const heatkv_config* cfg, const double* scas, const double* cas, int policy,
+                          int accounting, double b, const double* fraction, heatkv_schedule** out) {
+  if (!cfg || !out) return HEATKV_ERR_INVALID_ARG;
+  std::unique_ptr<heatkv_schedule> s(new (std::nothrow) heatkv_schedule);
+  if (!s) return HEATKV_ERR_HOST_MEMORY;
+  int rc;
+  try {
+    rc = build_schedule(*cfg, scas, cas, policy, accounting, b, fraction, &s->s);
+  } catch (const std::bad_alloc&) {
+    return HEATKV_ERR_HOST_MEMORY;
+  }
+  if (rc != HEATKV_OK) return rc;
+  *out = s.release();
+  return HEATKV_OK;
+}
+
+int heatkv_schedule_free(heatkv_schedule* sch) {
+  delete sch;
+  return HEATKV_OK;
+}
+
+int heatkv_schedule_masks(const heatkv_schedule* sch, uint16_t* attn_mask, uint16_t* keep_mask, int32_t* n_k,
+                          int64_t* budget_tokens) {
+  if (!sch) return HEATKV_ERR_INVALID_ARG;
+  const Schedule& s = sch->s;
+  if (attn_mask) std::memcpy(attn_mask, s.attn_mask.data(), s.attn_mask.size() * 2);
+  if (keep_mask) std::memcpy(keep_mask, s.keep_mask.data(), s.keep_mask.size() * 2);
+  if (n_k) std::memcpy(n_k, s.n_k.data(), s.n_k.size() * 4);
+  if (budget_tokens) *budget_tokens = s.budget;
+  return HEATKV_OK;
+}
+
+int heatkv_schedule_footprint(const heatkv_schedule* sch, int layout, int64_t* peak_tokens, int64_t* reserved_rows) {
+  if (!sch) return HEATKV_ERR_INVALID_ARG;
+  Plan plan;
+  int rc;
+  try {
+    rc = build_plan(sch->s, layout, &plan);
+  } catch (const std::bad_alloc&) {
+    return HEATKV_ERR_HOST_MEMORY;
+  }
+  if (rc != HEATKV_OK) return rc;
+  if (peak_tokens) *peak_tokens = plan.peak_tokens;
+  if (reserved_rows) *reserved_rows = plan.reserved_rows;
+  return HEATKV_OK;
+}
+
+int heatkv_schedule_plan(const heatkv_schedule* sch, int layout, int32_t* words, int64_t* n_words) {
+  if (!sch || !n_words) return HEATKV_ERR_INVALID_ARG;
+  Plan plan;
+  int rc;
+  try {
+    rc = build_plan(sch->s, layout, &plan);
+  } catch (const std::bad_alloc&) {
+    return HEATKV_ERR_HOST_MEMORY;
+  }
+  if (rc != HEATKV_OK) return rc;
+  if (words) {
+    if (*n_words < (int64_t)plan.blob.size()) return HEATKV_ERR_INVALID_ARG;
+    std::memcpy(words, plan.blob.data(), plan.blob.size() * 4);
+  }
+  *n_words = (int64_t)plan.blob.size();
+  return HEATKV_OK;
+}
+
+int heatkv_seq_open(heatkv_ctx* ctx, const heatkv_schedule* sch, void* stream_, int* seq_id) {
+  if (!ctx || !sch || !seq_id) return HEATKV_ERR_INVALID_ARG;
+  cudaStream_t stream = static_cast<cudaStream_t>(stream_);
+  int pi = -1, rc;
+  try {
+    rc = find_or_load_plan(ctx, sch->s, stream, &pi);
+  } catch (const std::bad_alloc&) {
+    return HEATKV_ERR_HOST_MEMORY;
+  }
+  if (rc != HEATKV_OK) return rc;
+  PlanEntry& pe = *ctx->plans[pi];
+  uint64_t start = 0;
+  if (!ctx->rows.alloc((uint64_t)pe.plan.reserved_rows, &start)) return HEATKV_ERR_OUT_OF_PAGES;
+  int id = -1;
+  for (size_t i = 0; i < ctx->seqs.size(); ++i)
+    if (!ctx->seqs[i].open) { id = (int)i; break; }
+  if (id < 0) { ctx->seqs.emplace_back(); id = (int)ctx->seqs.size() - 1; }
+  Seq& q = ctx->seqs[id];
+  q.open = true;
+  q.plan = pi;
+  q.base_row = start;
+  q.rows = (uint64_t)pe.plan.reserved_rows;
+  q.done_step.assign(ctx->cfg.L, -1);
+  q.pre_step.assign(ctx->cfg.L, -1);
+  pe.refs++;
+  ctx->reserved_rows += q.rows;
+  ctx->peak_reserved = std::max(ctx->peak_reserved, ctx->reserved_rows);
+  *seq_id = id;
+  return HEATKV_OK;
+}
+
+int heatkv_seq_close(heatkv_ctx* ctx, int seq_id) {
+  if (!ctx) return HEATKV_ERR_INVALID_ARG;
+  Seq* q = get_seq(ctx, seq_id);
+  if (!q) return HEATKV_ERR_INVALID_ARG;
+  ctx->rows.release(q->base_row, q->rows);
+  ctx->reserved_rows -= q->rows;
+  ctx->plans[q->plan]->refs--;
+  q->open = false;
+  return HEATKV_OK;
+}
+
+int heatkv_scale_attention(heatkv_ctx* ctx, const int* seq_ids, int n_seq, int layer, int step, const void* q,
+                           const void* k_new, const void* v_new, const heatkv_strides* st, const float* seg_bias,
+                           void* out, void* stream_) {
+  if (!ctx || !q || !k_new || !v_new || !out) return HEATKV_ERR_INVALID_ARG;
+  if (!aligned16(q) || !aligned16(k_new) || !aligned16(v_new) || !aligned16(out)) return HEATKV_ERR_INVALID_ARG;
+  cudaStream_t stream = static_cast<cudaStream_t>(stream_);
+  AttnParams p;
+  std::memset(&p, 0, sizeof(p));
+  int rc = gather_seqs(ctx, seq_ids, n_seq, layer, step, p.seqs);
+  if (rc != HEATKV_OK) return rc;
+  heatkv_strides s;
+  rc = check_strides(ctx, st, ctx->cfg.t[step], &s);
+  if (rc != HEATKV_OK) return rc;
+  fill_common(ctx, &p, s);
+  p.q = static_cast<const __nv_bfloat16*>(q);
+  p.k_new = static_cast<const __nv_bfloat16*>(k_new);
+  p.v_new = static_cast<const __nv_bfloat16*>(v_new);
+  p.out = static_cast<__nv_bfloat16*>(out);
+  p.seg_bias = seg_bias;
+  p.t_q = p.n_own = ctx->cfg.t[step];
+  p.step = step;
+  p.layer = layer;
+  const int choice = ctx->cfg.kernel;
+  bool use_tc = choice != HEATKV_KERNEL_GENERIC && tc_supported(ctx->tc, p, ctx->cfg.d, n_seq, false);
+  if (choice == HEATKV_KERNEL_AUTO && p.t_q < 256) use_tc = false;
+  cudaError_t e;
+  if (use_tc) {
+    int n = 0;
+    e = launch_attn_tc(ctx->tc, p, ctx->cfg.d, n_seq, false, stream, &n);
+    ctx->launches += n;
+  } else {
+    e = launch_attn_generic(p, ctx->cfg.d, n_seq, false, stream);
+    ctx->launches += 1;
+  }
+  return e == cudaSuccess ? HEATKV_OK : HEATKV_ERR_CUDA;
+}
+
+int heatkv_calibrate_scores(heatkv_ctx* ctx, int layer, int step, int n_seq, const void* q, const void* k_full,
+                            const void* v_full, const heatkv_strides* st, const float* seg_bias, float* beta_accum,
+                            void* out, void* stream_) {
+  if (!ctx || !q || !k_full || !beta_accum) return HEATKV_ERR_INVALID_ARG;
+  if (out && !v_full) return HEATKV_ERR_INVALID_ARG;
+  if (!aligned16(q) || !aligned16(k_full) || !aligned16(v_full) || !aligned16(out)) return HEATKV_ERR_INVALID_ARG;
+  if (layer < 0 || layer >= ctx->cfg.L || step < 0 || step >= ctx->cfg.K || n_seq < 1 || n_seq > 65535)
+    return HEATKV_ERR_INVALID_ARG;
+  cudaStream_t stream = static_cast<cudaStream_t>(stream_);
+  AttnParams p;
+  std::memset(&p, 0, sizeof(p));
+  heatkv_strides s;
+  if (!st) {   // dense: q/out [n_seq,H,t,d], k/v [n_seq,H,c[step],d]
+    const int64_t d = ctx->cfg.d, H = ctx->cfg.H, t = ctx->cfg.t[step], c = ctx->c[step];
+    s.q_tok = s.kv_tok = s.o_tok = d;
+    s.q_head = s.o_head = d * t; s.kv_head = d * c;
+    s.q_seq = s.o_seq = d * t * H; s.kv_seq = d * c * H;
+  } else {
+    int rc = check_strides(ctx, st, ctx->cfg.t[step], &s);
+    if (rc != HEATKV_OK) return rc;
+  }
+  fill_common(ctx, &p, s);
+  p.q = static_cast<const __nv_bfloat16*>(q);
+  p.k_new = static_cast<const __nv_bfloat16*>(k_full);
+  p.v_new = out ? static_cast<const __nv_bfloat16*>(v_full) : nullptr;
+  p.out = static_cast<__nv_bfloat16*>(out);
+  p.seg_bias = seg_bias;
+  p.t_q = ctx->cfg.t[step];
+  p.n_own = ctx->c[step];
+  p.step = step;
+  p.layer = layer;
+  p.beta_row = beta_accum + (((int64_t)layer * ctx->cfg.H) * ctx->cfg.K + step) * ctx->cfg.K;
+  cudaError_t e = launch_attn_generic(p, ctx->cfg.d, n_seq, true, stream);
+  ctx->launches += 1;
+  return e == cudaSuccess ? HEATKV_OK : HEATKV_ERR_CUDA;
+}
+
+int heatkv_finalize_scores(heatkv_ctx* ctx, const float* beta_accum, int n_samples, double* beta, double* scas,
+                           double* cas, void* stream_) {
+  if (!ctx || !beta_accum || n_samples < 1) return HEATKV_ERR_INVALID_ARG;
+  cudaStream_t stream = static_cast<cudaStream_t>(stream_);
+  const int L = ctx->cfg.L, H = ctx->cfg.H, K = ctx->cfg.K, s = ctx->cfg.s;
+  const size_t n = (size_t)L * H * K * K;
+  std::vector<float> host;
+  try {
+    host.resize(n);
+  } catch (const std::bad_alloc&) {
+    return HEATKV_ERR_HOST_MEMORY;
+  }
+  if (cudaMemcpyAsync(host.data(), beta_accum, n * 4, cudaMemcpyDeviceToHost, stream) != cudaSuccess)
+    return HEATKV_ERR_CUDA;
+  if (cudaStreamSynchronize(stream) != cudaSuccess) return HEATKV_ERR_CUDA;
+  for (size_t i = 0; i < n; ++i)
+    if (!std::isfinite(host[i])) return HEATKV_ERR_NAN_SCORE;
+  const double inv = 1.0 / (double)n_samples;
+  for (int hd = 0; hd < L * H; ++hd) {
+    const float* b = &host[(size_t)hd * K * K];
+    if (beta)
+      for (int i = 0; i < K * K; ++i) beta[(size_t)hd * K * K + i] = (double)b[i] * inv;
+    if (cas) {   // Eq. 3: last scale's mass on the cached non-sink scales, normaliser 1/(K-s)
+      double acc = 0.0;
+      for (int tau = s; tau <= K - 2; ++tau) acc += (double)b[(size_t)(K - 1) * K + tau] * inv;
+      cas[hd] = acc / (double)(K - s);
+    }
+    if (scas)    // Eq. 4: mean over the future scales tau > k of beta[tau][k], for s <= k <= K-2 (0-based)
+      for (int k = 0; k < K; ++k) {
+        double acc = 0.0;
+        if (k >= s && k <= K - 2) {
+          for (int tau = k + 1; tau < K; ++tau) acc += (double)b[(size_t)tau * K + k] * inv;
+          acc /= (double)(K - 1 - k);
+        }
+        scas[(size_t)hd * K + k] = acc;
+      }
+  }
+  return HEATKV_OK;
+}
+
+int heatkv_append_compact(heatkv_ctx* ctx, const int* seq_ids, int n_seq, int layer, int step, const void* k_new,
+                          const void* v_new, const heatkv_strides* st, void* stream_) {
+  if (!ctx || !seq_ids || n_seq < 1 || n_seq > HEATKV_MAX_BATCH) return HEATKV_ERR_INVALID_ARG;
+  if (step < 0 || step >= ctx->cfg.K || layer >= ctx->cfg.L) return HEATKV_ERR_INVALID_ARG;
+  if ((k_new == nullptr) != (v_new == nullptr)) return HEATKV_ERR_INVALID_ARG;
+  cudaStream_t stream = static_cast<cudaStream_t>(stream_);
+  const int L = ctx->cfg.L;
+  CopyParams p;
+  std::memset(&p, 0, sizeof(p));
+  p.k_pool = ctx->k_pool; p.v_pool = ctx->v_pool;
+  p.step = step; p.H = ctx->cfg.H; p.K = ctx->cfg.K; p.L = L; p.d = ctx->cfg.d;
+  p.t_k = ctx->cfg.t[step];
+
+  if (!k_new) {
+    // ---- eviction before the step starts (E_step)
+    const int l0 = layer < 0 ? 0 : layer, l1 = layer < 0 ? L : layer + 1;
+    bool moves = false;
+    for (int i = 0; i < n_seq; ++i) {
+      Seq* q = get_seq(ctx, seq_ids[i]);
+      if (!q) return HEATKV_ERR_INVALID_ARG;
+      for (int j = 0; j < i; ++j)
+        if (seq_ids[j] == seq_ids[i]) return HEATKV_ERR_INVALID_ARG;
+      for (int l = l0; l < l1; ++l)
+        if (q->done_step[l] != step - 1 || q->pre_step[l] >= step) return HEATKV_ERR_BAD_STEP_ORDER;
+      const PlanEntry& pe = *ctx->plans[q->plan];
+      p.seqs[i].plan = reinterpret_cast<const int32_t*>(ctx->meta + pe.meta_off);
+      p.seqs[i].base_row = (int64_t)q->base_row;
+      moves |= pe.plan.header().n_move > 0;
+    }
+    if (ctx->cfg.layout == HEATKV_LAYOUT_RAGGED && moves && step > 0) {
+      p.phase = 0; p.layer_begin = l0; p.n_layers = l1 - l0; p.layer = l0;
+      if (launch_compact(p, n_seq, stream) != cudaSuccess) return HEATKV_ERR_CUDA;
+      ctx->launches += 1;
+    }
+    for (int i = 0; i < n_seq; ++i)
+      for (int l = l0; l < l1; ++l) ctx->seqs[seq_ids[i]].pre_step[l] = (int16_t)step;
+    return HEATKV_OK;
+  }
+
+  // ---- update after the layer ran: drop G_step \ A_step of this layer, store the new scale
+  if (!aligned16(k_new) || !aligned16(v_new)) return HEATKV_ERR_INVALID_ARG;
+  int rc = gather_seqs(ctx, seq_ids, n_seq, layer, step, p.seqs);
+  if (rc != HEATKV_OK) return rc;
+  heatkv_strides s;
+  rc = check_strides(ctx, st, ctx->cfg.t[step], &s);
+  if (rc != HEATKV_OK) return rc;
+  p.kv_seq = s.kv_seq; p.kv_head = s.kv_head; p.kv_tok = s.kv_tok;
+  p.k_new = static_cast<const __nv_bfloat16*>(k_new);
+  p.v_new = static_cast<const __nv_bfloat16*>(v_new);
+  p.layer = layer;
+  if (step + 1 < ctx->cfg.K) {                  // the last scale is never cached
+    if (ctx->cfg.layout == HEATKV_LAYOUT_RAGGED) {
+      bool moves = false;
+      for (int i = 0; i < n_seq; ++i) moves |= ctx->plans[ctx->seqs[seq_ids[i]].plan]->plan.header().n_move > 0;
+      if (moves) {
+        p.phase = 1; p.layer_begin = layer; p.n_layers = 1;
+        if (launch_compact(p, n_seq, stream) != cudaSuccess) return HEATKV_ERR_CUDA;
+        ctx->launches += 1;
+      }
+    }
+    if (launch_append(p, n_seq, stream) != cudaSuccess) return HEATKV_ERR_CUDA;
+    ctx->launches += 1;
+  }
+  for (int i = 0; i < n_seq; ++i) ctx->seqs[seq_ids[i]].done_step[layer] = (int16_t)step;
+  return HEATKV_OK;
+}
+
+int heatkv_cache_bytes(heatkv_ctx* ctx, int seq_id, uint64_t* actual, uint64_t* reserved) {
+  if (!ctx) return HEATKV_ERR_INVALID_ARG;
+  Seq* q = get_seq(ctx, seq_id);
+  if (!q) return HEATKV_ERR_INVALID_ARG;
+  const Schedule& s = ctx->plans[q->plan]->sched;
+  uint64_t tokens = 0;
+  for (int l = 0; l < s.L; ++l)
+    for (int h = 0; h < s.H; ++h) {
+      uint16_t m = stored_mask(ctx, *q, l, h);
+      for (int i = 0; i < s.K; ++i)
+        if ((m >> i) & 1) tokens += s.t[i];
+    }
+  if (actual) *actual = tokens * ctx->cfg.d * 2 * 2;
+  if (reserved) *reserved = q->rows * ctx->cfg.d * 2 * 2;
+  return HEATKV_OK;
+}
+
+int heatkv_retained_indices(heatkv_ctx* ctx, int seq_id, int layer, int head, int32_t* idx, int* n) {
+  if (!ctx || !n) return HEATKV_ERR_INVALID_ARG;
+  Seq* q = get_seq(ctx, seq_id);
+  if (!q || layer < 0 || layer >= ctx->cfg.L || head < 0 || head >= ctx->cfg.H) return HEATKV_ERR_INVALID_ARG;
+  const Schedule& s = ctx->plans[q->plan]->sched;
+  uint16_t m = stored_mask(ctx, *q, layer, head);
+  int cnt = 0;
+  for (int i = 0; i < s.K; ++i)
+    if ((m >> i) & 1)
+      for (int j = 0; j < s.t[i]; ++j) {
+        if (idx) idx[cnt] = s.c[i] - s.t[i] + j;
+        ++cnt;
+      }
+  *n = cnt;
+  return HEATKV_OK;
+}
+
+int heatkv_export_head(heatkv_ctx* ctx, int seq_id, int layer, int head, void* k_out, void* v_out, void* stream_) {
+  if (!ctx || !k_out || !v_out) return HEATKV_ERR_INVALID_ARG;
+  Seq* q = get_seq(ctx, seq_id);
+  if (!q || layer < 0 || layer >= ctx->cfg.L || head < 0 || head >= ctx->cfg.H) return HEATKV_ERR_INVALID_ARG;
+  cudaStream_t stream = static_cast<cudaStream_t>(stream_);
+  const PlanEntry& pe = *ctx->plans[q->plan];
+  const Schedule& s = pe.sched;
+  const PlanHeader& h = pe.plan.header();
+  const int32_t* blob = pe.plan.blob.data();
+  const Desc* descs = reinterpret_cast<const Desc*>(blob + h.off_desc);
+  const uint16_t m = stored_mask(ctx, *q, layer, head);
+  const size_t row_bytes = (size_t)ctx->cfg.d * 2;
+  size_t out_row = 0;
+  int64_t dense = pe.plan.head_base[layer * s.H + head];
+  for (int i = 0; i < s.K; ++i) {
+    if (!((m >> i) & 1)) continue;
+    if (ctx->cfg.layout == HEATKV_LAYOUT_PAGED) {
+      // a head-scale keeps the rows it was appended to for its whole life
+      size_t u = s.at(i, layer, head);
+      const int32_t b0 = blob[h.off_app_begin + u], cnt = blob[h.off_app_cnt + u];
+      for (int j = 0; j < cnt; ++j) {
+        const Desc& dsc = descs[b0 + j];
+        const int nrow = dsc.meta & 0xff;
+        const int64_t row = (int64_t)q->base_row + dsc.row;
+        if (cudaMemcpyAsync(static_cast<char*>(k_out) + out_row * row_bytes, ctx->k_pool + row * ctx->cfg.d,
+                            nrow * row_bytes, cudaMemcpyDeviceToDevice, stream) != cudaSuccess ||
+            cudaMemcpyAsync(static_cast<char*>(v_out) + out_row * row_bytes, ctx->v_pool + row * ctx->cfg.d,
+                            nrow * row_bytes, cudaMemcpyDeviceToDevice, stream) != cudaSuccess)
+          return HEATKV_ERR_CUDA;
+        out_row += nrow;
+      }
+    } else {
+      const int64_t row = (int64_t)q->base_row + dense;
+      if (cudaMemcpyAsync(static_cast<char*>(k_out) + out_row * row_bytes, ctx->k_pool + row * ctx->cfg.d,
+                          s.t[i] * row_bytes, cudaMemcpyDeviceToDevice, stream) != cudaSuccess ||
+          cudaMemcpyAsync(static_cast<char*>(v_out) + out_row * row_bytes, ctx->v_pool + row * ctx->cfg.d,
+                          s.t[i] * row_bytes, cudaMemcpyDeviceToDevice, stream) != cudaSuccess)
+        return HEATKV_ERR_CUDA;
+      out_row += s.t[i];
+      dense += s.t[i];
+    }
+  }
+  return HEATKV_OK;
+}
+
+int heatkv_allocator_stats(heatkv_ctx* ctx, heatkv_alloc_stats* out) {
+  if (!ctx || !out) return HEATKV_ERR_INVALID_ARG;
+  std::memset(out, 0, sizeof(*out));
+  out->pool_rows = ctx->pool_rows;
+  out->reserved_rows = ctx->reserved_rows;
+  out->peak_reserved_rows = ctx->peak_reserved;
+  out->meta_bytes_used = ctx->meta_used;
+  for (size_t i = 0; i < ctx->seqs.size(); ++i)
+    if (ctx->seqs[i].open) {
+      out->open_seqs++;
+      uint64_t bytes = 0;
+      heatkv_cache_bytes(ctx, (int)i, &bytes, nullptr);
+      out->used_tokens += bytes / ((uint64_t)ctx->cfg.d * 4);
+    }
+  for (auto& pe : ctx->plans)
+    if (pe) out->plans++;
+  return HEATKV_OK;
+}
+
+int heatkv_launch_count(heatkv_ctx* ctx, uint64_t* n) {
+  if (!ctx || !n) return HEATKV_ERR_INVALID_ARG;
+  *n = ctx->launches;
+  return HEATKV_OK;
+}
+
+int heatkv_device_status(heatkv_ctx* ctx, void* stream_) {
+  if (!ctx) return HEATKV_ERR_INVALID_ARG;
+  cudaStream_t stream = static_cast<cudaStream_t>(stream_);
+  uint32_t word = 0;
+  if (cudaMemcpyAsync(&word, ctx->status, 4, cudaMemcpyDeviceToHost, stream) != cudaSuccess) return HEATKV_ERR_CUDA;
+  if (cudaStreamSynchronize(stream) != cudaSuccess) return HEATKV_ERR_CUDA;
+  return word == 0 ? HEATKV_OK : HEATKV_ERR_DEVICE_TIMEOUT;
+}
+
+}  // extern "C"

@@ -1,0 +1,357 @@
+// Generic ragged attention kernel (warp-level MMA, online softmax), used for the small,
+// bandwidth / latency bound scale steps and for calibration.
+//
+// One CTA = 64 queries of one (sequence, head); 4 warps x 16 query rows.  Keys arrive as a
+// sequence of half-tiles of up to 64 rows: first the head's retained prior keys, listed by
+// the plan's page table (Sec. 3.3: the head-scales not in A_k), then the step's own keys
+// from k_new.  In calibration mode (Eq. 2) every key comes from k_full and the per-row
+// probability mass of every source scale is accumulated next to the online softmax, so the
+// attention matrix alpha is never formed.
+#include "device_common.cuh"
+
+namespace heatkv {
+
+constexpr int GM = 64;    // queries per CTA
+constexpr int GN = 64;    // keys per half-tile
+constexpr int GTHREADS = 128;
+
+template <int D>
+struct GenericSmem {
+  static constexpr int TILE_BYTES = GN * D * 2;
+  // q | k[2] | v[2] | seg_sum[GM][16] | seg_ref[GM][16]
+  static constexpr int Q_OFF = 0;
+  static constexpr int K_OFF = GM * D * 2;
+  static constexpr int V_OFF = K_OFF + 2 * TILE_BYTES;
+  static constexpr int SEG_OFF = V_OFF + 2 * TILE_BYTES;
+  static constexpr int BYTES = SEG_OFF + 2 * GM * HEATKV_MAX_K * 4;
+};
+
+// byte offset of 16-byte chunk `ch` of row `r` in a [rows][D] bf16 tile (XOR swizzle)
+template <int D>
+__device__ __forceinline__ uint32_t tile_off(int r, int ch) {
+  return (uint32_t)((r * (D / 8) + (ch ^ (r & 7))) * 16);
+}
+
+// copies `rows` rows (row-major, D bf16 each, `stride` elements apart) into a swizzled tile;
+// rows >= n_valid are zero-filled.
+template <int D>
+__device__ __forceinline__ void load_tile(uint32_t smem_base, const __nv_bfloat16* src, int64_t stride,
+                                          int n_valid, int tid) {
+  constexpr int CH = D / 8;
+  constexpr int ROWS_PER_PASS = GTHREADS / CH;
+  const int ch = tid % CH;
+  const int r0 = tid / CH;
+#pragma unroll
+  for (int r = r0; r < GN; r += ROWS_PER_PASS) {
+    const bool ok = r < n_valid;
+    const __nv_bfloat16* p = ok ? src + (int64_t)r * stride + ch * 8 : src;
+    cp_async16(smem_base + tile_off<D>(r, ch), p, ok ? 16 : 0);
+  }
+}
+
+template <int D, bool CALIB>
+__global__ void __launch_bounds__(GTHREADS, 2) attn_generic_kernel(const __grid_constant__ AttnParams p) {
+  extern __shared__ __align__(128) unsigned char smem[];
+  using SM = GenericSmem<D>;
+  const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+  const int g = lane >> 2, qd = lane & 3;
+  const int seq = blockIdx.z;
+  const int q0 = blockIdx.x * GM;
+  int head = blockIdx.y;
+
+  const int2* descs = nullptr;
+  int n_desc = 0;
+  int64_t base_row = 0;
+  if (!CALIB) {
+    PlanView pv(p.seqs[seq].plan);
+    const int u = (p.step * p.L + p.layer) * p.H;
+    head = pv.order()[u + blockIdx.y];                   // heavy heads first
+    descs = pv.descs() + pv.attn_begin()[u + head];
+    n_desc = pv.attn_cnt()[u + head];
+    base_row = p.seqs[seq].base_row;
+  }
+  const int n_own_tiles = (p.n_own + GN - 1) / GN;
+  const int n_tiles = n_desc + n_own_tiles;
+
+  const uint32_t sbase = smem_u32(smem);
+  float* seg_sum = reinterpret_cast<float*>(smem + SM::SEG_OFF);
+  float* seg_ref = seg_sum + GM * HEATKV_MAX_K;
+
+  const __nv_bfloat16* kown = p.k_new + seq * p.kv_seq + head * p.kv_head;
+  const __nv_bfloat16* vown = p.v_new ? p.v_new + seq * p.kv_seq + head * p.kv_head : nullptr;
+
+  auto issue_tile = [&](int j, int stage) {
+    const __nv_bfloat16 *ks, *vs;
+    int64_t stride;
+    int nv;
+    if (j < n_desc) {
+      int2 dsc = descs[j];
+      int64_t row = base_row + dsc.x;
+      ks = p.k_pool + row * D;
+      vs = p.v_pool + row * D;
+      stride = D;
+      nv = dsc.y & 0xff;
+    } else {
+      int jj = j - n_desc;
+      ks = kown + (int64_t)jj * GN * p.kv_tok;
+      vs = vown ? vown + (int64_t)jj * GN * p.kv_tok : nullptr;
+      stride = p.kv_tok;
+      nv = min(GN, p.n_own - jj * GN);
+    }
+    load_tile<D>(sbase + SM::K_OFF + stage * SM::TILE_BYTES, ks, stride, nv, tid);
+    if (vs) load_tile<D>(sbase + SM::V_OFF + stage * SM::TILE_BYTES, vs, stride, nv, tid);
+  };
+
+  // ---- prologue: Q tile and the first key tile
+  {
+    const __nv_bfloat16* qsrc = p.q + seq * p.q_seq + head * p.q_head + (int64_t)q0 * p.q_tok;
+    load_tile<D>(sbase + SM::Q_OFF, qsrc, p.q_tok, min(GM, p.t_q - q0), tid);
+    cp_async_commit();
+    issue_tile(0, 0);
+    cp_async_commit();
+  }
+  if (CALIB) {
+    for (int i = tid; i < GM * HEATKV_MAX_K; i += GTHREADS) {
+      seg_sum[i] = 0.f;
+      seg_ref[i] = -INFINITY;
+    }
+  }
+  cp_async_wait<1>();
+  __syncthreads();
+
+  uint32_t qf[D / 16][4];
+#pragma unroll
+  for (int ks = 0; ks < D / 16; ++ks) {
+    int r = warp * 16 + (lane & 7) + ((lane >> 3) & 1) * 8;
+    int ch = ks * 2 + (lane >> 4);
+    ldmatrix_x4(qf[ks], sbase + SM::Q_OFF + tile_off<D>(r, ch));
+  }
+
+  float o[D / 8][4];
+#pragma unroll
+  for (int i = 0; i < D / 8; ++i) o[i][0] = o[i][1] = o[i][2] = o[i][3] = 0.f;
+  float m_run[2] = {-INFINITY, -INFINITY};
+  float l_run[2] = {0.f, 0.f};
+
+  for (int j = 0; j < n_tiles; ++j) {
+    const int stage = j & 1;
+    cp_async_wait<0>();
+    __syncthreads();                                   // tile j landed; everyone left tile j-1
+    if (j + 1 < n_tiles) issue_tile(j + 1, stage ^ 1);
+    cp_async_commit();
+
+    // tile attributes (warp-uniform)
+    int nv, seg_lo, seg_hi, col0 = 0;
+    if (j < n_desc) {
+      int2 dsc = descs[j];
+      nv = dsc.y & 0xff;
+      seg_lo = seg_hi = (dsc.y >> 8) & 0xff;
+    } else {
+      int jj = j - n_desc;
+      nv = min(GN, p.n_own - jj * GN);
+      col0 = jj * GN;
+      seg_lo = seg_hi = p.step;
+      if (CALIB) {
+        seg_lo = 0;
+        while (p.c[seg_lo] <= col0) ++seg_lo;
+        seg_hi = seg_lo;
+        while (p.c[seg_hi] < col0 + nv) ++seg_hi;
+      }
+    }
+
+    // ---- S = Q K^T
+    float s[GN / 8][4];
+#pragma unroll
+    for (int i = 0; i < GN / 8; ++i) s[i][0] = s[i][1] = s[i][2] = s[i][3] = 0.f;
+    const uint32_t kbase = sbase + SM::K_OFF + stage * SM::TILE_BYTES;
+#pragma unroll
+    for (int ks = 0; ks < D / 16; ++ks) {
+#pragma unroll
+      for (int np = 0; np < GN / 16; ++np) {
+        uint32_t b[4];
+        int r = np * 16 + (lane & 7) + (lane >> 4) * 8;
+        int ch = ks * 2 + ((lane >> 3) & 1);
+        ldmatrix_x4(b, kbase + tile_off<D>(r, ch));
+        mma_bf16(s[2 * np], qf[ks], b[0], b[1]);
+        mma_bf16(s[2 * np + 1], qf[ks], b[2], b[3]);
+      }
+    }
+
+    // ---- scale, bias, mask, online softmax
+    const float* bias_h = p.seg_bias ? p.seg_bias + head * p.K : nullptr;
+    const float LOG2E = 1.4426950408889634f;
+    float tile_bias = bias_h ? bias_h[seg_lo] * LOG2E : 0.f;
+    float mx[2] = {-INFINITY, -INFINITY};
+#pragma unroll
+    for (int n = 0; n < GN / 8; ++n) {
+#pragma unroll
+      for (int e = 0; e < 4; ++e) {
+        int col = n * 8 + qd * 2 + (e & 1);
+        float bias = tile_bias;
+        if (CALIB && bias_h && seg_lo != seg_hi) {
+          int sg = seg_lo;
+          while (p.c[sg] <= col0 + col && sg < seg_hi) ++sg;
+          bias = bias_h[sg] * LOG2E;
+        }
+        float v = col < nv ? fmaf(s[n][e], p.scale_log2, bias) : -INFINITY;
+        s[n][e] = v;
+        mx[e >> 1] = fmaxf(mx[e >> 1], v);
+      }
+    }
+    float corr[2];
+#pragma unroll
+    for (int r = 0; r < 2; ++r) {
+      mx[r] = fmaxf(mx[r], __shfl_xor_sync(0xffffffffu, mx[r], 1));
+      mx[r] = fmaxf(mx[r], __shfl_xor_sync(0xffffffffu, mx[r], 2));
+      float m_new = fmaxf(m_run[r], mx[r]);
+      corr[r] = exp2f(m_run[r] - m_new);
+      m_run[r] = m_new;
+      l_run[r] *= corr[r];
+    }
+    float psum[2] = {0.f, 0.f};
+#pragma unroll
+    for (int n = 0; n < GN / 8; ++n) {
+#pragma unroll
+      for (int e = 0; e < 4; ++e) {
+        float pv = exp2f(s[n][e] - m_run[e >> 1]);
+        s[n][e] = pv;
+        psum[e >> 1] += pv;
+      }
+    }
+    l_run[0] += psum[0];
+    l_run[1] += psum[1];
+
+    if (CALIB) {
+      // per-row mass of every source scale that intersects this tile, kept as (sum, reference max)
+      for (int sg = seg_lo; sg <= seg_hi; ++sg) {
+        const int lo = sg > 0 ? p.c[sg - 1] : 0, hi = p.c[sg];
+        float part[2] = {0.f, 0.f};
+#pragma unroll
+        for (int n = 0; n < GN / 8; ++n) {
+#pragma unroll
+          for (int e = 0; e < 4; ++e) {
+            int col = col0 + n * 8 + qd * 2 + (e & 1);
+            if (col >= lo && col < hi) part[e >> 1] += s[n][e];
+          }
+        }
+#pragma unroll
+        for (int r = 0; r < 2; ++r) {
+          part[r] += __shfl_xor_sync(0xffffffffu, part[r], 1);
+          part[r] += __shfl_xor_sync(0xffffffffu, part[r], 2);
+          if (qd == 0) {
+            int row = warp * 16 + g + r * 8;
+            float old = seg_sum[row * HEATKV_MAX_K + sg];
+            float ref = seg_ref[row * HEATKV_MAX_K + sg];
+            seg_sum[row * HEATKV_MAX_K + sg] = old * exp2f(ref - m_run[r]) + part[r];
+            seg_ref[row * HEATKV_MAX_K + sg] = m_run[r];
+          }
+        }
+      }
+    }
+
+    // ---- O = O * corr + P V
+    if (!CALIB || p.out) {
+#pragma unroll
+      for (int i = 0; i < D / 8; ++i) {
+        o[i][0] *= corr[0];
+        o[i][1] *= corr[0];
+        o[i][2] *= corr[1];
+        o[i][3] *= corr[1];
+      }
+      const uint32_t vbase = sbase + SM::V_OFF + stage * SM::TILE_BYTES;
+#pragma unroll
+      for (int kk = 0; kk < GN / 16; ++kk) {
+        uint32_t pa[4];
+        pa[0] = pack_bf16(s[2 * kk][0], s[2 * kk][1]);
+        pa[1] = pack_bf16(s[2 * kk][2], s[2 * kk][3]);
+        pa[2] = pack_bf16(s[2 * kk + 1][0], s[2 * kk + 1][1]);
+        pa[3] = pack_bf16(s[2 * kk + 1][2], s[2 * kk + 1][3]);
+#pragma unroll
+        for (int dp = 0; dp < D / 16; ++dp) {
+          uint32_t b[4];
+          int r = kk * 16 + (lane & 7) + ((lane >> 3) & 1) * 8;
+          int ch = dp * 2 + (lane >> 4);
+          ldmatrix_x4_trans(b, vbase + tile_off<D>(r, ch));
+          mma_bf16(o[2 * dp], pa, b[0], b[1]);
+          mma_bf16(o[2 * dp + 1], pa, b[2], b[3]);
+        }
+      }
+    }
+  }
+  cp_async_wait<0>();
+
+  // ---- epilogue
+  float inv_l[2];
+#pragma unroll
+  for (int r = 0; r < 2; ++r) {
+    float l = l_run[r];
+    l += __shfl_xor_sync(0xffffffffu, l, 1);
+    l += __shfl_xor_sync(0xffffffffu, l, 2);
+    inv_l[r] = 1.f / l;
+  }
+
+  if (CALIB) {
+    // beta[step][sg] += (1/t) * sum over rows of mass(row, sg) / l(row)     (Eq. 2)
+    float* beta = p.beta_row + (int64_t)head * p.K * p.K;
+    for (int sg = 0; sg <= p.step; ++sg) {
+      float acc = 0.f;
+      if (qd == 0) {
+#pragma unroll
+        for (int r = 0; r < 2; ++r) {
+          int row = warp * 16 + g + r * 8;
+          if (q0 + row < p.t_q)
+            acc += seg_sum[row * HEATKV_MAX_K + sg] * exp2f(seg_ref[row * HEATKV_MAX_K + sg] - m_run[r]) * inv_l[r];
+        }
+      }
+      acc += __shfl_xor_sync(0xffffffffu, acc, 4);
+      acc += __shfl_xor_sync(0xffffffffu, acc, 8);
+      acc += __shfl_xor_sync(0xffffffffu, acc, 16);
+      if (lane == 0) atomicAdd(beta + sg, acc / (float)p.t_q);
+    }
+  }
+
+  if (p.out) {
+    __syncthreads();                                   // all warps are done with the K/V stages
+    // stage the bf16 tile in shared memory (reusing the Q region), then 16-byte row stores
+#pragma unroll
+    for (int n = 0; n < D / 8; ++n) {
+      int r0 = warp * 16 + g;
+      uint32_t lo = pack_bf16(o[n][0] * inv_l[0], o[n][1] * inv_l[0]);
+      uint32_t hi = pack_bf16(o[n][2] * inv_l[1], o[n][3] * inv_l[1]);
+      *reinterpret_cast<uint32_t*>(smem + SM::Q_OFF + tile_off<D>(r0, n) + qd * 4) = lo;
+      *reinterpret_cast<uint32_t*>(smem + SM::Q_OFF + tile_off<D>(r0 + 8, n) + qd * 4) = hi;
+    }
+    __syncthreads();
+    constexpr int CH = D / 8;
+    __nv_bfloat16* dst = p.out + seq * p.o_seq + head * p.o_head + (int64_t)q0 * p.o_tok;
+    for (int i = tid; i < GM * CH; i += GTHREADS) {
+      int r = i / CH, ch = i % CH;
+      if (q0 + r < p.t_q) {
+        int4 v = *reinterpret_cast<const int4*>(smem + SM::Q_OFF + tile_off<D>(r, ch));
+        *reinterpret_cast<int4*>(dst + (int64_t)r * p.o_tok + ch * 8) = v;
+      }
+    }
+  }
+}
+
+template <int D, bool CALIB>
+static cudaError_t launch_one(const AttnParams& p, int n_seq, cudaStream_t stream) {
+  auto kern = attn_generic_kernel<D, CALIB>;
+  static bool configured = false;
+  if (!configured) {
+    cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, GenericSmem<D>::BYTES);
+    if (e != cudaSuccess) return e;
+    configured = true;
+  }
+  dim3 grid((p.t_q + GM - 1) / GM, p.H, n_seq);
+  kern<<<grid, GTHREADS, GenericSmem<D>::BYTES, stream>>>(p);
+  return cudaGetLastError();
+}
+
+cudaError_t launch_attn_generic(const AttnParams& p, int d, int n_seq, bool calib, cudaStream_t stream) {
+  if (d == 128) return calib ? launch_one<128, true>(p, n_seq, stream) : launch_one<128, false>(p, n_seq, stream);
+  if (d == 64) return calib ? launch_one<64, true>(p, n_seq, stream) : launch_one<64, false>(p, n_seq, stream);
+  return cudaErrorInvalidValue;
+}
+
+}  // namespace heatkv

@@ -1,0 +1,76 @@
+// Internal host-side declarations shared by the translation units of libheatkv.
+#pragma once
+#include <cstdint>
+#include <vector>
+
+#include "heatkv.h"
+
+namespace heatkv {
+
+// ---------------------------------------------------------------- schedule (host)
+struct Schedule {
+  int L = 0, H = 0, K = 0, s = 0;
+  int t[HEATKV_MAX_K] = {0};
+  int c[HEATKV_MAX_K] = {0};             // c[i] = t[0] + .. + t[i]
+  int policy = 0;
+  int64_t budget = -1;                   // B in tokens, -1 for EXPLICIT
+  std::vector<int32_t> n_k;              // [K]
+  std::vector<uint16_t> attn_mask;       // [K][L][H]
+  std::vector<uint16_t> keep_mask;       // [K][L][H]
+  uint64_t uid = 0;                      // identity used to cache plans per context
+  size_t at(int step, int l, int h) const { return ((size_t)step * L + l) * H + h; }
+};
+
+// ---------------------------------------------------------------- plan (host image of device tables)
+// One key half-tile: up to 64 consecutive pool rows that belong to one source scale.
+struct Desc {
+  int32_t row;      // row relative to the sequence's reservation
+  int32_t meta;     // n_valid (bits 0..7) | source scale (bits 8..15)
+};
+// One in-place move of the ragged layout: n rows from src to dst (dst < src), relative rows.
+struct Move {
+  int32_t src, dst, n, pad;
+};
+
+// Offsets (in 4-byte words from the start of the blob) of the tables of a plan.  The blob
+// is what lives in the metadata region; kernels receive its device address.
+struct PlanHeader {
+  int32_t L, H, K, n_desc;
+  int32_t off_desc;        // Desc[n_desc]
+  int32_t off_attn_begin;  // int32[K*L*H] first desc of the visible prior keys
+  int32_t off_attn_cnt;    // int32[K*L*H]
+  int32_t off_app_begin;   // int32[K*L*H] first desc of the rows the step's K/V go to
+  int32_t off_app_cnt;     // int32[K*L*H] 0 = the head does not store this scale
+  int32_t off_order;       // int32[K*L*H] heads of a (step, layer) sorted by visible keys, descending
+  int32_t off_move;        // Move[n_move]
+  int32_t off_pre_begin;   // int32[K*L*H] moves of the eviction before the step   (ragged)
+  int32_t off_pre_cnt;
+  int32_t off_post_begin;  // int32[K*L*H] moves of the eviction after the layer   (ragged)
+  int32_t off_post_cnt;
+  int32_t n_move;
+  int32_t total_words;
+  int32_t pad[3];
+};
+static_assert(sizeof(PlanHeader) % 16 == 0, "header must keep 16-byte alignment");
+
+struct Plan {
+  int layout = 0;
+  int64_t reserved_rows = 0;            // multiple of HEATKV_PAGE_TOKENS
+  int64_t peak_tokens = 0;
+  std::vector<int32_t> blob;            // PlanHeader followed by the tables
+  // host-only bookkeeping for introspection -------------------------------------------------
+  // place[(l*H+h)*K + i] = first relative row of source scale i in the paged layout (-1: never stored)
+  std::vector<int32_t> place;
+  // ragged: base row and capacity of every head
+  std::vector<int32_t> head_base, head_cap;
+  // tokens cached after the pre-step eviction of step k / after layer l of step k
+  std::vector<int64_t> tokens_pre;      // [K]
+  std::vector<int64_t> tokens_post;     // [K][L]
+  const PlanHeader& header() const { return *reinterpret_cast<const PlanHeader*>(blob.data()); }
+};
+
+int build_schedule(const heatkv_config& cfg, const double* scas, const double* cas, int policy,
+                   int accounting, double b, const double* fraction, Schedule* out);
+int build_plan(const Schedule& sch, int layout, Plan* out);
+
+}  // namespace heatkv

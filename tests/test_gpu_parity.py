@@ -1,0 +1,232 @@
+"""GPU parity: the CUDA path (through the C ABI) against the CPU oracle on the same seeded
+inputs.  Retained indices and cache contents bit-exact; attention within max-abs 1e-2 and
+mean-abs 1e-3; calibration scores within 1e-3 relative."""
+import math
+
+import numpy as np
+import pytest
+import torch
+
+import heatkv_workloads as W
+from oracle import heatkv_oracle as O
+
+pytestmark = pytest.mark.gpu
+
+ATOL_MAX, ATOL_MEAN, RTOL_BETA = 1e-2, 1e-3, 1e-3
+
+
+@pytest.fixture(scope="module")
+def hk():
+    import paper_2605_14877_b200 as hk
+    return hk
+
+
+def _session(hk, sh, pool_rows, layout, kernel=None, **kw):
+    from paper_2605_14877_b200.sweep import Session
+    return Session(sh.L, sh.H, sh.d, sh.t, sh.s, pool_rows, layout=layout,
+                   kernel=hk.KERNEL_GENERIC if kernel is None else kernel, **kw)
+
+
+def _f64(x):
+    return O.bf16_bits_to_f64(W.bf16_bits(x))
+
+
+def _check_attention(got_bf16, ref_f64, what):
+    got = got_bf16.to(torch.float64).cpu().numpy()
+    err = np.abs(got - ref_f64)
+    assert err.max() <= ATOL_MAX, (what, err.max())
+    assert err.mean() <= ATOL_MEAN, (what, err.mean())
+
+
+def _run_full_parity(hk, sh, ref, make_schedule, layout, seed=0, bias=None, kernel=None, n_seq=None,
+                     check_heads=None, check_cache=True):
+    """Whole generation of one batch; compares every (seq, layer, head, step) unless check_heads
+    restricts the oracle work to a list of (seq, layer, head)."""
+    n_seq = sh.n_seq if n_seq is None else n_seq
+    sm = 1.0 / math.sqrt(sh.d)
+    with _session(hk, sh, pool_rows=n_seq * (sh.L * sh.H * (sh.c[-2] + 64 * sh.K) + 64), layout=layout,
+                  kernel=kernel) as ses:
+        sch = make_schedule(ses)
+        ids = [hk.heatkv_seq_open(ses.ctx, sch) for _ in range(n_seq)]
+        layers = [W.qkv_layer(sh, seed, l, device="cuda", n_seq=n_seq) for l in range(sh.L)]
+        outs = [torch.zeros_like(layers[l][0]) for l in range(sh.L)]
+        host = [[_f64(x) for x in layers[l]] for l in range(sh.L)]
+        bits = [[W.bf16_bits(x) for x in layers[l][1:]] for l in range(sh.L)]
+        bias_dev = None if bias is None else torch.from_numpy(bias).cuda()
+        heads = check_heads or [(s_, l, h) for s_ in range(n_seq) for l in range(sh.L) for h in range(sh.H)]
+
+        def after(step, layer):
+            if not check_cache or step + 1 >= sh.K:
+                return
+            for (s_, l, h) in heads:
+                if l != layer:
+                    continue
+                idx, kk, vv = O.cache_after_layer(bits[l][0][s_, h], bits[l][1][s_, h], ref, step + 1, l, h)
+                got_idx = hk.heatkv_retained_indices(ses.ctx, ids[s_], l, h, sh.c[-1])
+                assert np.array_equal(got_idx, idx), (step, l, h)
+                ko = torch.zeros(max(len(idx), 1), sh.d, dtype=torch.bfloat16, device="cuda")
+                vo = torch.zeros_like(ko)
+                hk.heatkv_export_head(ses.ctx, ids[s_], l, h, ko, vo)
+                assert np.array_equal(W.bf16_bits(ko)[: len(idx)], kk), (step, l, h)
+                assert np.array_equal(W.bf16_bits(vo)[: len(idx)], vv), (step, l, h)
+
+        ses.generate(ids, lambda l: layers[l], lambda l: outs[l],
+                     (lambda l, k: bias_dev[l, k]) if bias is not None else None, after)
+        torch.cuda.synchronize()
+        assert hk.heatkv_device_status(ses.ctx) == 0
+        for (s_, l, h) in heads:
+            q, k, v = host[l]
+            for step in range(1, sh.K + 1):
+                lo, hi = (sh.c[step - 2] if step > 1 else 0), sh.c[step - 1]
+                brow = None if bias is None else bias[l, step - 1, h].astype(np.float64)
+                want = O.scale_attention(q[s_, h, lo:hi], k[s_, h], v[s_, h], ref, step, l, h, sm, brow)
+                _check_attention(outs[l][s_, h, lo:hi], want, (s_, l, h, step))
+        # closed form of the cache size at the end (last stored scale is K-1)
+        kept = O.kept_tokens_after_step(ref, sh.K - 1)
+        actual, reserved = hk.heatkv_cache_bytes(ses.ctx, ids[0])
+        assert actual == O.cache_bytes(kept, sh.d) and reserved >= actual
+        st = hk.heatkv_allocator_stats(ses.ctx)
+        assert st.open_seqs == n_seq and st.used_tokens == n_seq * int(kept.sum())
+        for i in ids:
+            hk.heatkv_seq_close(ses.ctx, i)
+        assert hk.heatkv_allocator_stats(ses.ctx).reserved_rows == 0
+        launches = hk.heatkv_launch_count(ses.ctx)
+        hk.heatkv_schedule_free(sch)
+    return launches
+
+
+@pytest.mark.parametrize("layout", [0, 1], ids=["ragged", "paged"])
+def test_tiny_config_end_to_end(hk, layout):
+    """Config 1: 1 layer, 4 heads, d=64, sides {1,2,4,8}, per-head budgets {100,50,25,0} %."""
+    sh = W.TINY
+    frac = np.array([W.TINY_FRACTIONS])
+    ref = O.explicit_schedule(frac, sh.s, sh.sides)
+    n = _run_full_parity(hk, sh, ref, lambda ses: ses.schedule(policy=hk.POLICY_EXPLICIT, fraction=frac), layout)
+    assert n >= sh.K
+
+
+@pytest.mark.parametrize("layout", [0, 1], ids=["ragged", "paged"])
+@pytest.mark.parametrize("policy", [0, 1, 2], ids=["heatkv", "binary", "naive"])
+def test_mid_config_multi_layer_with_bias(hk, layout, policy):
+    """d=128, 3 layers, 11 scales (several key tiles, ragged tails 36/144/400), per-head logit bias."""
+    sh = W.Shape("mid", L=3, H=4, d=128, sides=W.SIDES_13[:11], n_seq=2, s=3)
+    scores = W.synthetic_scas(sh, 4)
+    cas = scores[:, :, 6].copy()
+    ref = O.heatkv_schedule(cas if policy == 1 else scores, 0.15, sh.s, sh.sides, policy)
+    bias = W.seg_bias_prior_lognormal(sh, 3)
+    _run_full_parity(hk, sh, ref, lambda ses: ses.schedule(scas=scores, cas=cas, policy=policy, b=0.15), layout,
+                     bias=bias)
+
+
+def test_full_budget_equals_uncompressed(hk):
+    sh = W.Shape("full", L=1, H=2, d=64, sides=W.SIDES_13[:9], n_seq=1, s=2)
+    scores = W.synthetic_scas(sh, 1)
+    ref = O.heatkv_schedule(scores, 1.0, sh.s, sh.sides)
+    _run_full_parity(hk, sh, ref, lambda ses: ses.schedule(scas=scores, b=1.0), hk.LAYOUT_PAGED)
+
+
+def _calibrate(hk, sh, seeds, bias=None, with_out=False):
+    from paper_2605_14877_b200.sweep import Session
+    sm = 1.0 / math.sqrt(sh.d)
+    ses = Session(sh.L, sh.H, sh.d, sh.t, sh.s, pool_rows=64, kernel=hk.KERNEL_GENERIC)
+    beta_dev = torch.zeros(sh.L, sh.H, sh.K, sh.K, dtype=torch.float32, device="cuda")
+    bias_dev = None if bias is None else torch.from_numpy(bias).cuda()
+    ref = np.zeros((sh.L, sh.H, sh.K, sh.K))
+    n_samples = 0
+    for seed in seeds:
+        for l in range(sh.L):
+            q, k, v = W.qkv_layer(sh, seed, l, device="cuda")
+            out = torch.zeros_like(q) if with_out else None
+            for step in range(sh.K):
+                lo, hi = ses.step_slices(step)
+                qs, ks, vs = q[:, :, lo:hi], k[:, :, :hi], v[:, :, :hi]
+                os_ = out[:, :, lo:hi] if with_out else None
+                st = hk.Strides.of(qs, ks, os_)
+                hk.heatkv_calibrate_scores(ses.ctx, l, step, sh.n_seq, qs, ks, vs if with_out else None, st,
+                                           None if bias is None else bias_dev[l, step], beta_dev, os_)
+            qh, kh, vh = _f64(q), _f64(k), _f64(v)
+            for s_ in range(sh.n_seq):
+                for h in range(sh.H):
+                    b_lh = None if bias is None else bias[l, :, h, :].astype(np.float64)
+                    ref[l, h] += O.beta_sample(qh[s_, h], kh[s_, h], sh.sides, sm, b_lh)
+            if with_out:
+                full = O.explicit_schedule(np.ones((sh.L, sh.H)), sh.s, sh.sides)
+                for h in range(sh.H):
+                    for step in range(1, sh.K + 1):
+                        lo, hi = (sh.c[step - 2] if step > 1 else 0), sh.c[step - 1]
+                        brow = None if bias is None else bias[l, step - 1, h].astype(np.float64)
+                        want = O.scale_attention(qh[0, h, lo:hi], kh[0, h], vh[0, h], full, step, l, h, sm, brow)
+                        _check_attention(out[0, h, lo:hi], want, ("calib-out", l, h, step))
+        n_samples += sh.n_seq
+    beta, scas, cas = hk.heatkv_finalize_scores(ses.ctx, beta_dev, n_samples, sh.L, sh.H, sh.K)
+    ses.close()
+    ref /= n_samples
+    return beta, scas, cas, ref
+
+
+def test_calibration_tiny_four_samples(hk):
+    sh = W.TINY
+    beta, scas, cas, ref = _calibrate(hk, sh, seeds=range(4))
+    assert np.allclose(beta.sum(axis=-1), 1.0, atol=2e-4)
+    assert np.all(np.triu(beta, 1) == 0)
+    mask = ref > 1e-6
+    assert np.all(np.abs(beta - ref)[mask] <= RTOL_BETA * ref[mask])
+    for l in range(sh.L):
+        for h in range(sh.H):
+            assert np.allclose(scas[l, h], O.scas(ref[l, h], sh.s), rtol=RTOL_BETA, atol=1e-9)
+            assert np.isclose(cas[l, h], O.cas(ref[l, h], sh.s), rtol=RTOL_BETA, atol=1e-9)
+
+
+def test_calibration_mid_with_bias_and_output(hk):
+    sh = W.Shape("mid", L=2, H=3, d=128, sides=W.SIDES_13[:10], n_seq=2, s=3)
+    bias = W.seg_bias_prior_lognormal(sh, 8)
+    beta, scas, cas, ref = _calibrate(hk, sh, seeds=[5], bias=bias, with_out=True)
+    mask = ref > 1e-5
+    assert np.all(np.abs(beta - ref)[mask] <= RTOL_BETA * ref[mask])
+    assert np.allclose(beta.sum(axis=-1), 1.0, atol=2e-4)
+    for l in range(sh.L):
+        for h in range(sh.H):
+            assert np.allclose(scas[l, h], O.scas(ref[l, h], sh.s), rtol=RTOL_BETA, atol=1e-9)
+
+
+def test_config2_sampled_heads(hk):
+    """Config 2 (2B single layer, 16 heads, d=128, 13 scales, batch 2, 20x) at full size in the
+    launch configuration the bench times; the oracle checks a sample of (seq, head) pairs."""
+    sh = W.CFG2
+    scores = W.synthetic_scas(sh, 0)
+    ref = O.heatkv_schedule(scores, 0.05, sh.s, sh.sides)
+    bias = W.seg_bias_current_scale(sh, 0)
+    heads = [(0, 0, 0), (1, 0, 5), (0, 0, 11), (1, 0, 15)]
+    _run_full_parity(hk, sh, ref, lambda ses: ses.schedule(scas=scores, b=0.05), hk.LAYOUT_PAGED, bias=bias,
+                     kernel=hk.KERNEL_AUTO, check_heads=heads)
+
+
+def test_step_order_and_pool_errors(hk):
+    sh = W.Shape("err", L=2, H=2, d=64, sides=W.SIDES_13[:8], n_seq=1, s=1)
+    scores = W.synthetic_scas(sh, 2)
+    from paper_2605_14877_b200.sweep import Session
+    ses = Session(sh.L, sh.H, sh.d, sh.t, sh.s, pool_rows=1024)
+    sch = ses.schedule(scas=scores, b=1.0)
+    # full cache of this shape needs more rows than the pool has
+    with pytest.raises(hk.HeatKVError) as e:
+        hk.heatkv_seq_open(ses.ctx, sch)
+    assert e.value.status == -4
+    sch2 = ses.schedule(scas=scores, b=0.1)
+    sid = hk.heatkv_seq_open(ses.ctx, sch2)
+    q, k, v = W.qkv_layer(sh, 0, 0, device="cuda")
+    out = torch.zeros_like(q)
+    with pytest.raises(hk.HeatKVError) as e:            # step 1 before step 0
+        ses.run_layer_step([sid], 0, 1, q, k, v, out)
+    assert e.value.status == -5
+    ses.run_layer_step([sid], 0, 0, q, k, v, out)
+    with pytest.raises(hk.HeatKVError) as e:            # same step twice
+        ses.run_layer_step([sid], 0, 0, q, k, v, out)
+    assert e.value.status == -5
+    with pytest.raises(hk.HeatKVError):                 # unknown sequence
+        ses.run_layer_step([sid + 7], 0, 1, q, k, v, out)
+    with pytest.raises(hk.HeatKVError):                 # misaligned pointer
+        hk.heatkv_scale_attention(ses.ctx, [sid], 1, 0, q.data_ptr() + 2, k, v, None, None, out)
+    hk.heatkv_seq_close(ses.ctx, sid)
+    hk.heatkv_schedule_free(sch)
+    hk.heatkv_schedule_free(sch2)
+    ses.close()
