@@ -53,13 +53,19 @@ class ClockSampler:
     """Samples SM clocks and throttle reasons with nvidia-smi while the timed region runs."""
     Q = ("clocks.sm,clocks.max.sm,clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
          "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
+    Q_OLD = Q.replace("clocks_event_reasons", "clocks_throttle_reasons")
 
     def __init__(self, index: int):
         self.index, self.proc, self.lines = index, None, []
 
     def start(self):
         try:
-            self.proc = subprocess.Popen(["nvidia-smi", f"--id={self.index}", f"--query-gpu={self.Q}",
+            query = self.Q
+            probe = subprocess.run(["nvidia-smi", f"--id={self.index}", f"--query-gpu={query}",
+                                    "--format=csv,noheader,nounits"], capture_output=True, text=True, timeout=30)
+            if probe.returncode != 0 or "not a valid" in (probe.stdout + probe.stderr).lower():
+                query = self.Q_OLD
+            self.proc = subprocess.Popen(["nvidia-smi", f"--id={self.index}", f"--query-gpu={query}",
                                           "--format=csv,noheader,nounits", "-lms", "100"],
                                          stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
             self.thread = threading.Thread(target=self._read, daemon=True)

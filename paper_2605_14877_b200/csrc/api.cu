@@ -422,6 +422,7 @@ int heatkv_scale_attention(heatkv_ctx* ctx, const int* seq_ids, int n_seq, int l
   const int choice = ctx->cfg.kernel;
   bool use_tc = choice != HEATKV_KERNEL_GENERIC && tc_supported(ctx->tc, p, ctx->cfg.d, n_seq, false);
   if (choice == HEATKV_KERNEL_AUTO && p.t_q < 256) use_tc = false;
+  if (choice == HEATKV_KERNEL_TCGEN05 && !use_tc) return HEATKV_ERR_INVALID_ARG;   // never a silent substitute
   cudaError_t e;
   if (use_tc) {
     int n = 0;

@@ -1,14 +1,569 @@
-// Tensor-memory attention kernel for the large scale steps (placeholder translation unit:
-// reports "unsupported" until the tcgen05 path is linked in).
+// Tensor-memory attention kernel for the large scale steps (head_dim 128).
+//
+// One CTA owns 256 queries of one (sequence, head) as two 128-row tiles A and B that share
+// the key/value stream.  Warp roles:
+//   warp 0      TMA producer: Q tiles once, then K and V half-tiles (64 rows x 128 dims each)
+//               gathered through the plan's page table, followed by the step's own keys.
+//   warp 1      MMA issuer: S = Q K^T and O += P V with tcgen05.mma, accumulators in TMEM.
+//   warps 4-7   softmax of tile A, warps 8-11 softmax of tile B: one thread per query row
+//               reads its row of S from TMEM, keeps the running max / sum, writes P (bf16)
+//               back into the columns S occupied, and rescales O only when the row max grew
+//               by more than 2^8 since the last reference (the sum keeps the same reference,
+//               so the result is exact).
+// TMEM columns: S_A/P_A 0..127, S_B/P_B 128..255, O_A 256..383, O_B 384..511.
+// The MMA order S_A S_B (PV_A S_A' PV_B S_B')* lets the softmax of one tile overlap the
+// tensor work of the other.  Every wait is bounded; on expiry the CTA records a status word,
+// drains its own copies and leaves.
+#include <cuda.h>
+#include <cudaTypedefs.h>
+
 #include "device_common.cuh"
 #include "internal.h"
 
 namespace heatkv {
-struct TcState {};
-int tc_create(const heatkv_config&, void*, void*, uint64_t, TcState** out) { *out = nullptr; return HEATKV_OK; }
-void tc_destroy(TcState*) {}
-bool tc_supported(const TcState*, const AttnParams&, int, int, bool) { return false; }
-cudaError_t launch_attn_tc(TcState*, const AttnParams&, int, int, bool, cudaStream_t, int*) {
-  return cudaErrorNotSupported;
+
+namespace tc {
+
+constexpr int D = 128;
+constexpr int BM = 128;                 // rows per Q tile
+constexpr int BN = 128;                 // keys per tile (two 64-row half-tiles)
+constexpr int HALF = 64;
+constexpr int THREADS = 384;
+constexpr int KV_STAGES = 2;
+constexpr uint32_t HALF_COLS_BYTES = 128 * 128;        // one 64-column half of a 128-row tile: 16 KB
+constexpr uint32_t TILE_BYTES = 2 * HALF_COLS_BYTES;   // 32 KB
+constexpr uint32_t SLOT_BYTES = HALF * 128;            // 64 rows x 128 B inside one column half
+
+// shared memory map (bytes from a 1024-aligned base)
+constexpr uint32_t SM_Q = 0;                                   // 2 tiles
+constexpr uint32_t SM_K = SM_Q + 2 * TILE_BYTES;               // KV_STAGES tiles
+constexpr uint32_t SM_V = SM_K + KV_STAGES * TILE_BYTES;       // KV_STAGES tiles
+constexpr uint32_t SM_BAR = SM_V + KV_STAGES * TILE_BYTES;     // barriers + scalars
+constexpr uint32_t SM_TOTAL = SM_BAR + 256;
+constexpr uint32_t SM_ALLOC = SM_TOTAL + 1024;                 // slack for manual alignment
+
+// barrier slots (8 bytes each) inside SM_BAR
+enum Bar : uint32_t {
+  Q_FULL = 0,                   // +x (2)
+  K_FULL = 2, K_EMPTY = 4,      // +stage
+  V_FULL = 6, V_EMPTY = 8,      // +stage
+  S_FULL = 10,                  // +x  S_x of tile j is in TMEM
+  P_FULL = 12,                  // +x  P_x of tile j is in TMEM (128 arrivals)
+  PV_DONE = 14,                 // +x  O_x includes tile j
+  N_BARS = 16
+};
+constexpr uint32_t SM_TMEM_PTR = SM_BAR + N_BARS * 8;
+constexpr uint32_t SM_ABORT = SM_TMEM_PTR + 4;
+
+constexpr uint32_t WAIT_LIMIT = 1u << 20;               // about a second with the hint below
+constexpr float RESCALE_THRESHOLD = 8.0f;               // log2 units
+
+__device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
+  asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count));
 }
+__device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes) {
+  asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ void mbar_arrive(uint32_t bar) {
+  asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
+}
+__device__ __forceinline__ bool mbar_try(uint32_t bar, uint32_t parity) {
+  uint32_t ok;
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2, %3;\n\t"
+      "selp.u32 %0, 1, 0, p;\n\t}"
+      : "=r"(ok)
+      : "r"(bar), "r"(parity), "r"(1000u)            // suspend-time hint: about a microsecond per try
+      : "memory");
+  return ok != 0;
+}
+// Bounded wait.  Returns false when the CTA is aborting (this wait or another one ran out).
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile uint32_t* abort_flag,
+                                          uint32_t* status) {
+  for (uint32_t it = 0; it < WAIT_LIMIT; ++it) {
+    if (mbar_try(bar, parity)) return true;
+    if ((it & 31u) == 31u && *abort_flag) return false;
+  }
+  *abort_flag = 1;
+  atomicOr(status, 1u);
+  return false;
+}
+
+__device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap* map, int c0, int c1, uint32_t bar) {
+  asm volatile(
+      "cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];"
+      ::"r"(dst), "l"(map), "r"(c0), "r"(c1), "r"(bar)
+      : "memory");
+}
+__device__ __forceinline__ void tma_load_4d(uint32_t dst, const CUtensorMap* map, int c0, int c1, int c2, int c3,
+                                            uint32_t bar) {
+  asm volatile(
+      "cp.async.bulk.tensor.4d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3, %4, %5}], [%6];"
+      ::"r"(dst), "l"(map), "r"(c0), "r"(c1), "r"(c2), "r"(c3), "r"(bar)
+      : "memory");
+}
+
+__device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void tc_commit(uint32_t bar) {
+  asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
+}
+// D(tmem) (+)= A(smem desc) * B(smem desc)
+__device__ __forceinline__ void mma_ss(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc, uint32_t idesc, uint32_t acc) {
+  asm volatile(
+      "{\n\t.reg .pred p;\n\tsetp.ne.b32 p, %4, 0;\n\t"
+      "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}"
+      ::"r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(acc)
+      : "memory");
+}
+// D(tmem) (+)= A(tmem) * B(smem desc)
+__device__ __forceinline__ void mma_ts(uint32_t d_tmem, uint32_t a_tmem, uint64_t b_desc, uint32_t idesc, uint32_t acc) {
+  asm volatile(
+      "{\n\t.reg .pred p;\n\tsetp.ne.b32 p, %4, 0;\n\t"
+      "tcgen05.mma.cta_group::1.kind::f16 [%0], [%1], %2, %3, p;\n\t}"
+      ::"r"(d_tmem), "r"(a_tmem), "l"(b_desc), "r"(idesc), "r"(acc)
+      : "memory");
+}
+__device__ __forceinline__ void tmem_ld32(uint32_t taddr, uint32_t (&r)[32]) {
+  asm volatile(
+      "tcgen05.ld.sync.aligned.32x32b.x32.b32 "
+      "{%0,%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15,"
+      "%16,%17,%18,%19,%20,%21,%22,%23,%24,%25,%26,%27,%28,%29,%30,%31}, [%32];"
+      : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]),
+        "=r"(r[8]), "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15]),
+        "=r"(r[16]), "=r"(r[17]), "=r"(r[18]), "=r"(r[19]), "=r"(r[20]), "=r"(r[21]), "=r"(r[22]), "=r"(r[23]),
+        "=r"(r[24]), "=r"(r[25]), "=r"(r[26]), "=r"(r[27]), "=r"(r[28]), "=r"(r[29]), "=r"(r[30]), "=r"(r[31])
+      : "r"(taddr)
+      : "memory");
+}
+__device__ __forceinline__ void tmem_st32(uint32_t taddr, const uint32_t (&r)[32]) {
+  asm volatile(
+      "tcgen05.st.sync.aligned.32x32b.x32.b32 [%0], "
+      "{%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15,%16,"
+      "%17,%18,%19,%20,%21,%22,%23,%24,%25,%26,%27,%28,%29,%30,%31,%32};"
+      ::"r"(taddr), "r"(r[0]), "r"(r[1]), "r"(r[2]), "r"(r[3]), "r"(r[4]), "r"(r[5]), "r"(r[6]), "r"(r[7]),
+        "r"(r[8]), "r"(r[9]), "r"(r[10]), "r"(r[11]), "r"(r[12]), "r"(r[13]), "r"(r[14]), "r"(r[15]),
+        "r"(r[16]), "r"(r[17]), "r"(r[18]), "r"(r[19]), "r"(r[20]), "r"(r[21]), "r"(r[22]), "r"(r[23]),
+        "r"(r[24]), "r"(r[25]), "r"(r[26]), "r"(r[27]), "r"(r[28]), "r"(r[29]), "r"(r[30]), "r"(r[31])
+      : "memory");
+}
+__device__ __forceinline__ void tmem_st16(uint32_t taddr, const uint32_t (&r)[16]) {
+  asm volatile(
+      "tcgen05.st.sync.aligned.32x32b.x16.b32 [%0], "
+      "{%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15,%16};"
+      ::"r"(taddr), "r"(r[0]), "r"(r[1]), "r"(r[2]), "r"(r[3]), "r"(r[4]), "r"(r[5]), "r"(r[6]), "r"(r[7]),
+        "r"(r[8]), "r"(r[9]), "r"(r[10]), "r"(r[11]), "r"(r[12]), "r"(r[13]), "r"(r[14]), "r"(r[15])
+      : "memory");
+}
+__device__ __forceinline__ void tmem_wait_ld() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
+__device__ __forceinline__ void tmem_wait_st() { asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory"); }
+
+// Shared-memory matrix descriptor, 128-byte swizzle, descriptor version 1.
+__device__ __forceinline__ uint64_t smem_desc(uint32_t addr, uint32_t lbo_bytes, uint32_t sbo_bytes) {
+  return (uint64_t)((addr >> 4) & 0x3FFFu) | ((uint64_t)((lbo_bytes >> 4) & 0x3FFFu) << 16) |
+         ((uint64_t)((sbo_bytes >> 4) & 0x3FFFu) << 32) | (1ull << 46) | (2ull << 61);
+}
+// kind::f16 instruction descriptor: D fp32, A/B bf16, M x N.
+__host__ __device__ constexpr uint32_t instr_desc(int M, int N, int a_mn_major, int b_mn_major) {
+  return (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)a_mn_major << 15) | ((uint32_t)b_mn_major << 16) |
+         ((uint32_t)(N >> 3) << 17) | ((uint32_t)(M >> 4) << 24);
+}
+
+struct Maps {
+  CUtensorMap q, k_own, v_own, k_pool, v_pool;
+};
+
+// One key half-tile: where it comes from and how many of its 64 rows are real.
+struct Slot {
+  int pool_row;     // >= 0: row in the pool; < 0: own-scale tokens starting at -(pool_row + 1)
+  int n_valid;
+  int seg;
+};
+
+__device__ __forceinline__ Slot get_slot(int i, const int2* descs, int n_desc, int n_slots, int64_t base_row,
+                                         int t_own, int step) {
+  Slot s;
+  int valid = i < n_slots;
+  if (!valid) i = n_slots - 1;                      // padding half-tile: re-read finite data, mask everything
+  if (i < n_desc) {
+    int2 d = descs[i];
+    s.pool_row = (int)(base_row + d.x);
+    s.n_valid = d.y & 0xff;
+    s.seg = (d.y >> 8) & 0xff;
+  } else {
+    int tok0 = (i - n_desc) * HALF;
+    s.pool_row = -(tok0 + 1);
+    s.n_valid = min(HALF, t_own - tok0);
+    s.seg = step;
+  }
+  if (!valid) s.n_valid = 0;
+  return s;
+}
+
+__global__ void __launch_bounds__(THREADS, 1)
+attn_tc_kernel(const __grid_constant__ AttnParams p, const __grid_constant__ Maps maps) {
+  extern __shared__ unsigned char smem_raw[];
+  const uint32_t raw = smem_u32(smem_raw);
+  const uint32_t sbase = (raw + 1023u) & ~1023u;
+  unsigned char* sgen = smem_raw + (sbase - raw);
+  volatile uint32_t* abort_flag = reinterpret_cast<volatile uint32_t*>(sgen + SM_ABORT);
+  volatile uint32_t* tmem_ptr_smem = reinterpret_cast<volatile uint32_t*>(sgen + SM_TMEM_PTR);
+  auto bar = [&](uint32_t which) { return sbase + SM_BAR + which * 8; };
+
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int seq = blockIdx.z;
+  const int q0 = blockIdx.x * (2 * BM);
+  const int nq = (q0 + BM < p.t_q) ? 2 : 1;          // does tile B hold any query?
+
+  PlanView pv(p.seqs[seq].plan);
+  const int u = (p.step * p.L + p.layer) * p.H;
+  const int head = pv.order()[u + blockIdx.y];
+  const int2* descs = pv.descs() + pv.attn_begin()[u + head];
+  const int n_desc = pv.attn_cnt()[u + head];
+  const int64_t base_row = p.seqs[seq].base_row;
+  const int n_slots = n_desc + (p.n_own + HALF - 1) / HALF;
+  const int n_tiles = (n_slots + 1) / 2;
+
+  if (threadIdx.x == 0) {
+    *abort_flag = 0;
+    mbar_init(bar(Q_FULL + 0), 1);
+    mbar_init(bar(Q_FULL + 1), 1);
+    for (int s = 0; s < KV_STAGES; ++s) {
+      mbar_init(bar(K_FULL + s), 1);
+      mbar_init(bar(K_EMPTY + s), 1);
+      mbar_init(bar(V_FULL + s), 1);
+      mbar_init(bar(V_EMPTY + s), 1);
+    }
+    for (int x = 0; x < 2; ++x) {
+      mbar_init(bar(S_FULL + x), 1);
+      mbar_init(bar(P_FULL + x), BM);
+      mbar_init(bar(PV_DONE + x), 1);
+    }
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+  }
+  if (warp == 0) {
+    __syncwarp();
+    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(sbase + SM_TMEM_PTR), "r"(512u)
+                 : "memory");
+    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+  }
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  const uint32_t tmem = *tmem_ptr_smem;
+
+  if (warp == 0) {
+    // ------------------------------------------------------------------ TMA producer
+    if (lane == 0) {
+      uint32_t armed_k = 0, armed_v = 0;               // stage -> a copy was issued at least once
+      uint32_t par_k[KV_STAGES] = {0, 0}, par_v[KV_STAGES] = {0, 0};
+      for (int x = 0; x < nq; ++x) {
+        mbar_expect_tx(bar(Q_FULL + x), TILE_BYTES);
+        for (int ch = 0; ch < 2; ++ch)
+          for (int hf = 0; hf < 2; ++hf)
+            tma_load_4d(sbase + SM_Q + x * TILE_BYTES + ch * HALF_COLS_BYTES + hf * SLOT_BYTES, &maps.q, ch * 64,
+                        q0 + x * BM + hf * HALF, head, seq, bar(Q_FULL + x));
+      }
+      bool ok = true;
+      for (int j = 0; j < n_tiles && ok; ++j) {
+        const int st = j % KV_STAGES;
+        const uint32_t use = (uint32_t)(j / KV_STAGES);
+        Slot sl[2];
+        for (int hf = 0; hf < 2; ++hf) sl[hf] = get_slot(2 * j + hf, descs, n_desc, n_slots, base_row, p.n_own, p.step);
+        // K first: the S product of the next tile needs it earliest
+        if (use > 0) ok = mbar_wait(bar(K_EMPTY + st), (use - 1) & 1, abort_flag, p.status);
+        if (!ok) break;
+        mbar_expect_tx(bar(K_FULL + st), TILE_BYTES);
+        armed_k |= 1u << st;
+        par_k[st] = use & 1;
+        for (int hf = 0; hf < 2; ++hf)
+          for (int ch = 0; ch < 2; ++ch) {
+            uint32_t dst = sbase + SM_K + st * TILE_BYTES + ch * HALF_COLS_BYTES + hf * SLOT_BYTES;
+            if (sl[hf].pool_row >= 0) tma_load_2d(dst, &maps.k_pool, ch * 64, sl[hf].pool_row, bar(K_FULL + st));
+            else tma_load_4d(dst, &maps.k_own, ch * 64, -sl[hf].pool_row - 1, head, seq, bar(K_FULL + st));
+          }
+        if (use > 0) ok = mbar_wait(bar(V_EMPTY + st), (use - 1) & 1, abort_flag, p.status);
+        if (!ok) break;
+        mbar_expect_tx(bar(V_FULL + st), TILE_BYTES);
+        armed_v |= 1u << st;
+        par_v[st] = use & 1;
+        for (int hf = 0; hf < 2; ++hf)
+          for (int ch = 0; ch < 2; ++ch) {
+            uint32_t dst = sbase + SM_V + st * TILE_BYTES + ch * HALF_COLS_BYTES + hf * SLOT_BYTES;
+            if (sl[hf].pool_row >= 0) tma_load_2d(dst, &maps.v_pool, ch * 64, sl[hf].pool_row, bar(V_FULL + st));
+            else tma_load_4d(dst, &maps.v_own, ch * 64, -sl[hf].pool_row - 1, head, seq, bar(V_FULL + st));
+          }
+      }
+      if (!ok) {
+        // leaving early: let every copy this thread started land before the CTA exits
+        for (int s = 0; s < KV_STAGES; ++s) {
+          if (armed_k & (1u << s))
+            for (uint32_t it = 0; it < WAIT_LIMIT && !mbar_try(bar(K_FULL + s), par_k[s]); ++it) {}
+          if (armed_v & (1u << s))
+            for (uint32_t it = 0; it < WAIT_LIMIT && !mbar_try(bar(V_FULL + s), par_v[s]); ++it) {}
+        }
+        for (int x = 0; x < nq; ++x)
+          for (uint32_t it = 0; it < WAIT_LIMIT && !mbar_try(bar(Q_FULL + x), 0); ++it) {}
+      }
+    }
+  } else if (warp == 1) {
+    // ------------------------------------------------------------------ MMA issuer
+    if (lane == 0) {
+      constexpr uint32_t IDESC_S = instr_desc(BM, BN, 0, 0);     // Q, K both K-major
+      constexpr uint32_t IDESC_PV = instr_desc(BM, D, 0, 1);     // P from TMEM, V MN-major
+      bool ok = true;
+      auto issue_s = [&](int x, int st) {
+        const uint32_t qa = sbase + SM_Q + x * TILE_BYTES, ka = sbase + SM_K + st * TILE_BYTES;
+#pragma unroll
+        for (int ks = 0; ks < D / 16; ++ks) {
+          const uint32_t off = (ks >> 2) * HALF_COLS_BYTES + (ks & 3) * 32;
+          mma_ss(tmem + x * 128, smem_desc(qa + off, 16, 1024), smem_desc(ka + off, 16, 1024), IDESC_S, ks > 0);
+        }
+      };
+      auto issue_pv = [&](int x, int st, bool first) {
+        const uint32_t va = sbase + SM_V + st * TILE_BYTES;
+#pragma unroll
+        for (int ks = 0; ks < BN / 16; ++ks)
+          mma_ts(tmem + 256 + x * 128, tmem + x * 128 + ks * 8, smem_desc(va + ks * 2048, HALF_COLS_BYTES, 1024),
+                 IDESC_PV, !(first && ks == 0));
+      };
+      for (int x = 0; x < nq && ok; ++x) ok = mbar_wait(bar(Q_FULL + x), 0, abort_flag, p.status);
+      if (ok) ok = mbar_wait(bar(K_FULL + 0), 0, abort_flag, p.status);
+      if (ok) {
+        tc_fence_after();
+        for (int x = 0; x < nq; ++x) {
+          issue_s(x, 0);
+          tc_commit(bar(S_FULL + x));
+        }
+        tc_commit(bar(K_EMPTY + 0));
+      }
+      for (int j = 0; j < n_tiles && ok; ++j) {
+        const int st = j % KV_STAGES, stn = (j + 1) % KV_STAGES;
+        const uint32_t par = (uint32_t)(j / KV_STAGES) & 1, parn = (uint32_t)((j + 1) / KV_STAGES) & 1;
+        const bool more = j + 1 < n_tiles;
+        ok = mbar_wait(bar(V_FULL + st), par, abort_flag, p.status);
+        if (ok && more) ok = mbar_wait(bar(K_FULL + stn), parn, abort_flag, p.status);
+        for (int x = 0; x < nq && ok; ++x) {
+          ok = mbar_wait(bar(P_FULL + x), j & 1, abort_flag, p.status);
+          if (!ok) break;
+          tc_fence_after();
+          issue_pv(x, st, j == 0);
+          tc_commit(bar(PV_DONE + x));
+          if (more) {
+            issue_s(x, stn);
+            tc_commit(bar(S_FULL + x));
+          }
+        }
+        if (ok) {
+          tc_commit(bar(V_EMPTY + st));
+          if (more) tc_commit(bar(K_EMPTY + stn));
+        }
+      }
+    }
+  } else if (warp >= 4) {
+    // ------------------------------------------------------------------ softmax + epilogue
+    const int x = (warp - 4) >> 2;                      // 0: tile A, 1: tile B
+    if (x < nq) {
+      const int row = (warp & 3) * 32 + lane;           // row inside the tile == TMEM lane
+      const uint32_t lane_base = (uint32_t)((warp & 3) * 32) << 16;
+      const uint32_t t_s = tmem + lane_base + x * 128;
+      const uint32_t t_o = tmem + lane_base + 256 + x * 128;
+      const float* bias_h = p.seg_bias ? p.seg_bias + head * p.K : nullptr;
+      const float LOG2E = 1.4426950408889634f;
+      float m_ref = -INFINITY, l_sum = 0.f;
+      bool ok = true;
+      for (int j = 0; j < n_tiles && ok; ++j) {
+        Slot s0 = get_slot(2 * j, descs, n_desc, n_slots, base_row, p.n_own, p.step);
+        Slot s1 = get_slot(2 * j + 1, descs, n_desc, n_slots, base_row, p.n_own, p.step);
+        const float b0 = bias_h ? bias_h[s0.seg] * LOG2E : 0.f;
+        const float b1 = bias_h ? bias_h[s1.seg] * LOG2E : 0.f;
+        ok = __all_sync(0xffffffffu, mbar_wait(bar(S_FULL + x), j & 1, abort_flag, p.status));
+        if (!ok) break;
+        tc_fence_after();
+        // pass 1: row maximum of the scaled, biased, masked logits
+        float mx = -INFINITY;
+#pragma unroll
+        for (int c = 0; c < 4; ++c) {
+          uint32_t r[32];
+          tmem_ld32(t_s + c * 32, r);
+          tmem_wait_ld();
+          const int nv = (c < 2 ? s0.n_valid : s1.n_valid) - (c & 1) * 32;
+          const float bb = c < 2 ? b0 : b1;
+#pragma unroll
+          for (int i = 0; i < 32; ++i) {
+            float v = fmaf(__uint_as_float(r[i]), p.scale_log2, bb);
+            mx = fmaxf(mx, i < nv ? v : -INFINITY);
+          }
+        }
+        const float m_new = fmaxf(m_ref, mx);
+        const bool grow = m_new > m_ref + RESCALE_THRESHOLD;   // also true on the first tile (m_ref = -inf)
+        if (j > 0 && __any_sync(0xffffffffu, grow)) {
+          // O_x holds tiles < j relative to m_ref: rescale the rows whose reference moves
+          ok = __all_sync(0xffffffffu, mbar_wait(bar(PV_DONE + x), (j - 1) & 1, abort_flag, p.status));
+          if (!ok) break;
+          tc_fence_after();
+          const float f = grow ? exp2f(m_ref - m_new) : 1.f;
+#pragma unroll
+          for (int c = 0; c < 4; ++c) {
+            uint32_t r[32];
+            tmem_ld32(t_o + c * 32, r);
+            tmem_wait_ld();
+#pragma unroll
+            for (int i = 0; i < 32; ++i) r[i] = __float_as_uint(__uint_as_float(r[i]) * f);
+            tmem_st32(t_o + c * 32, r);
+          }
+          tmem_wait_st();
+          l_sum *= f;
+        }
+        if (grow) m_ref = m_new;
+        // pass 2: p = exp2(logit - m_ref), row sum in fp32, P as bf16 pairs into the S columns
+#pragma unroll
+        for (int c = 0; c < 4; ++c) {
+          uint32_t r[32];
+          tmem_ld32(t_s + c * 32, r);
+          tmem_wait_ld();
+          const int nv = (c < 2 ? s0.n_valid : s1.n_valid) - (c & 1) * 32;
+          const float bb = (c < 2 ? b0 : b1) - m_ref;
+          uint32_t pk[16];
+#pragma unroll
+          for (int i = 0; i < 32; i += 2) {
+            float e0 = i < nv ? exp2f(fmaf(__uint_as_float(r[i]), p.scale_log2, bb)) : 0.f;
+            float e1 = i + 1 < nv ? exp2f(fmaf(__uint_as_float(r[i + 1]), p.scale_log2, bb)) : 0.f;
+            l_sum += e0 + e1;
+            pk[i >> 1] = pack_bf16(e0, e1);
+          }
+          // chunk c covers keys 32c..32c+31 -> P columns 16c..16c+15.  Column 16c+15 <= 32c+31 has
+          // been read already for every c, so writing never clobbers unread logits.
+          tmem_st16(t_s + c * 16, pk);
+        }
+        tmem_wait_st();
+        tc_fence_before();
+        mbar_arrive(bar(P_FULL + x));
+      }
+      if (ok) ok = __all_sync(0xffffffffu, mbar_wait(bar(PV_DONE + x), (n_tiles - 1) & 1, abort_flag, p.status));
+      if (ok) {
+        tc_fence_after();
+        const float inv = 1.f / l_sum;
+        const bool live = q0 + x * BM + row < p.t_q;
+        __nv_bfloat16* dst = p.out + seq * p.o_seq + head * p.o_head + (int64_t)(q0 + x * BM + row) * p.o_tok;
+#pragma unroll
+        for (int c = 0; c < 4; ++c) {
+          uint32_t r[32];
+          tmem_ld32(t_o + c * 32, r);
+          tmem_wait_ld();
+          if (live) {
+#pragma unroll
+            for (int i = 0; i < 32; i += 8) {
+              int4 v;
+              v.x = (int)pack_bf16(__uint_as_float(r[i]) * inv, __uint_as_float(r[i + 1]) * inv);
+              v.y = (int)pack_bf16(__uint_as_float(r[i + 2]) * inv, __uint_as_float(r[i + 3]) * inv);
+              v.z = (int)pack_bf16(__uint_as_float(r[i + 4]) * inv, __uint_as_float(r[i + 5]) * inv);
+              v.w = (int)pack_bf16(__uint_as_float(r[i + 6]) * inv, __uint_as_float(r[i + 7]) * inv);
+              *reinterpret_cast<int4*>(dst + c * 32 + i) = v;
+            }
+          }
+        }
+      }
+    }
+  }
+
+  tc_fence_before();
+  __syncthreads();
+  if (warp == 0) {
+    tc_fence_after();
+    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem), "r"(512u) : "memory");
+  }
+}
+
+}  // namespace tc
+
+// ---------------------------------------------------------------------------------- host side
+struct TcState {
+  PFN_cuTensorMapEncodeTiled_v12000 encode = nullptr;
+  CUtensorMap k_pool, v_pool;
+  bool ready = false;
+};
+
+namespace {
+
+bool encode_2d(TcState* st, CUtensorMap* m, void* base, uint64_t rows) {
+  cuuint64_t dims[2] = {(cuuint64_t)tc::D, (cuuint64_t)rows};
+  cuuint64_t strides[1] = {(cuuint64_t)tc::D * 2};
+  cuuint32_t box[2] = {64, (cuuint32_t)tc::HALF};
+  cuuint32_t estr[2] = {1, 1};
+  return st->encode(m, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, base, dims, strides, box, estr,
+                    CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                    CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
+// [n_seq, H, t, d] view with element strides -> 4-D map (d, token, head, sequence)
+bool encode_4d(TcState* st, CUtensorMap* m, const void* base, int t, int H, int n_seq, int64_t s_tok, int64_t s_head,
+               int64_t s_seq) {
+  cuuint64_t dims[4] = {(cuuint64_t)tc::D, (cuuint64_t)t, (cuuint64_t)H, (cuuint64_t)n_seq};
+  // a stride of 0 is not encodable; a dimension of extent 1 may carry any positive stride
+  auto fix = [](int64_t s) { return (cuuint64_t)((s > 0 ? s : 8) * 2); };
+  cuuint64_t strides[3] = {fix(s_tok), fix(s_head), fix(s_seq)};
+  cuuint32_t box[4] = {64, (cuuint32_t)tc::HALF, 1, 1};
+  cuuint32_t estr[4] = {1, 1, 1, 1};
+  return st->encode(m, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 4, const_cast<void*>(base), dims, strides, box, estr,
+                    CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                    CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
+}  // namespace
+
+int tc_create(const heatkv_config& cfg, void* k_pool, void* v_pool, uint64_t pool_rows, TcState** out) {
+  *out = nullptr;
+  TcState* st = new (std::nothrow) TcState;
+  if (!st) return HEATKV_ERR_HOST_MEMORY;
+  *out = st;
+  if (cfg.d != tc::D) return HEATKV_OK;                 // only head_dim 128 runs on this path
+  void* fn = nullptr;
+  cudaDriverEntryPointQueryResult qres;
+  if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &fn, cudaEnableDefault, &qres) != cudaSuccess ||
+      qres != cudaDriverEntryPointSuccess || !fn) {
+    cudaGetLastError();
+    return HEATKV_OK;                                   // no driver entry point: generic kernel only
+  }
+  st->encode = reinterpret_cast<PFN_cuTensorMapEncodeTiled_v12000>(fn);
+  if (!encode_2d(st, &st->k_pool, k_pool, pool_rows) || !encode_2d(st, &st->v_pool, v_pool, pool_rows))
+    return HEATKV_OK;
+  if (cudaFuncSetAttribute(tc::attn_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)tc::SM_ALLOC) !=
+      cudaSuccess) {
+    cudaGetLastError();
+    return HEATKV_OK;
+  }
+  st->ready = true;
+  return HEATKV_OK;
+}
+
+void tc_destroy(TcState* st) { delete st; }
+
+bool tc_supported(const TcState* st, const AttnParams& p, int d, int n_seq, bool calib) {
+  if (!st || !st->ready || calib || d != tc::D || n_seq > 65535) return false;
+  // TMA needs 16-byte aligned bases (checked by the caller) and strides that are multiples of 16 bytes
+  const int64_t s[6] = {p.q_seq, p.q_head, p.q_tok, p.kv_seq, p.kv_head, p.kv_tok};
+  for (int64_t v : s)
+    if (v & 7) return false;
+  return true;
+}
+
+cudaError_t launch_attn_tc(TcState* st, const AttnParams& p, int d, int n_seq, bool calib, cudaStream_t stream,
+                           int* launches) {
+  (void)d; (void)calib;
+  tc::Maps maps;
+  maps.k_pool = st->k_pool;
+  maps.v_pool = st->v_pool;
+  if (!encode_4d(st, &maps.q, p.q, p.t_q, p.H, n_seq, p.q_tok, p.q_head, p.q_seq) ||
+      !encode_4d(st, &maps.k_own, p.k_new, p.n_own, p.H, n_seq, p.kv_tok, p.kv_head, p.kv_seq) ||
+      !encode_4d(st, &maps.v_own, p.v_new, p.n_own, p.H, n_seq, p.kv_tok, p.kv_head, p.kv_seq))
+    return cudaErrorInvalidValue;
+  dim3 grid((p.t_q + 2 * tc::BM - 1) / (2 * tc::BM), p.H, n_seq);
+  tc::attn_tc_kernel<<<grid, tc::THREADS, tc::SM_ALLOC, stream>>>(p, maps);
+  *launches = 1;
+  return cudaGetLastError();
+}
+
 }  // namespace heatkv
