@@ -156,6 +156,24 @@ __device__ __forceinline__ void tmem_st16(uint32_t taddr, const uint32_t (&r)[16
         "r"(r[8]), "r"(r[9]), "r"(r[10]), "r"(r[11]), "r"(r[12]), "r"(r[13]), "r"(r[14]), "r"(r[15])
       : "memory");
 }
+__device__ __forceinline__ float fmax3(float a, float b, float c) {
+  float d;
+  asm("max.f32 %0, %1, %2, %3;" : "=f"(d) : "f"(a), "f"(b), "f"(c));
+  return d;
+}
+__device__ __forceinline__ float ex2_approx(float x) {
+  float y;
+  asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
+  return y;
+}
+template <uint32_t N>
+__device__ __forceinline__ void reg_alloc() {
+  asm volatile("setmaxnreg.inc.sync.aligned.u32 %0;" ::"n"(N));
+}
+template <uint32_t N>
+__device__ __forceinline__ void reg_dealloc() {
+  asm volatile("setmaxnreg.dec.sync.aligned.u32 %0;" ::"n"(N));
+}
 __device__ __forceinline__ void tmem_wait_ld() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
 __device__ __forceinline__ void tmem_wait_st() { asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory"); }
 
@@ -254,6 +272,9 @@ attn_tc_kernel(const __grid_constant__ AttnParams p, const __grid_constant__ Map
   tc_fence_after();
   const uint32_t tmem = *tmem_ptr_smem;
 
+  // register budget per warpgroup: 128*72 + 256*216 <= 64K
+  if (warp < 4) {
+    reg_dealloc<72>();
   if (warp == 0) {
     // ------------------------------------------------------------------ TMA producer
     if (lane == 0) {
@@ -362,7 +383,9 @@ attn_tc_kernel(const __grid_constant__ AttnParams p, const __grid_constant__ Map
         }
       }
     }
-  } else if (warp >= 4) {
+  }
+  } else {
+    reg_alloc<216>();
     // ------------------------------------------------------------------ softmax + epilogue
     const int x = (warp - 4) >> 2;                      // 0: tile A, 1: tile B
     if (x < nq) {
@@ -382,21 +405,31 @@ attn_tc_kernel(const __grid_constant__ AttnParams p, const __grid_constant__ Map
         ok = __all_sync(0xffffffffu, mbar_wait(bar(S_FULL + x), j & 1, abort_flag, p.status));
         if (!ok) break;
         tc_fence_after();
-        // pass 1: row maximum of the scaled, biased, masked logits
-        float mx = -INFINITY;
-#pragma unroll
-        for (int c = 0; c < 4; ++c) {
-          uint32_t r[32];
-          tmem_ld32(t_s + c * 32, r);
-          tmem_wait_ld();
-          const int nv = (c < 2 ? s0.n_valid : s1.n_valid) - (c & 1) * 32;
-          const float bb = c < 2 ? b0 : b1;
+        // whole row of S into registers (one wait for the four loads)
+        uint32_t r0[32], r1[32], r2[32], r3[32];
+        tmem_ld32(t_s, r0);
+        tmem_ld32(t_s + 32, r1);
+        tmem_ld32(t_s + 64, r2);
+        tmem_ld32(t_s + 96, r3);
+        tmem_wait_ld();
+        if (s0.n_valid < HALF || s1.n_valid < HALF) {            // ragged tile (warp-uniform): mask by -inf
 #pragma unroll
           for (int i = 0; i < 32; ++i) {
-            float v = fmaf(__uint_as_float(r[i]), p.scale_log2, bb);
-            mx = fmaxf(mx, i < nv ? v : -INFINITY);
+            if (i >= s0.n_valid) r0[i] = 0xff800000u;
+            if (i + 32 >= s0.n_valid) r1[i] = 0xff800000u;
+            if (i >= s1.n_valid) r2[i] = 0xff800000u;
+            if (i + 32 >= s1.n_valid) r3[i] = 0xff800000u;
           }
         }
+        // row maximum: the logit is raw * scale + bias(half) with scale > 0, so take the raw maxima
+        float mx0 = fmaxf(__uint_as_float(r0[0]), __uint_as_float(r1[0]));
+        float mx1 = fmaxf(__uint_as_float(r2[0]), __uint_as_float(r3[0]));
+#pragma unroll
+        for (int i = 1; i < 32; ++i) {
+          mx0 = fmax3(mx0, __uint_as_float(r0[i]), __uint_as_float(r1[i]));
+          mx1 = fmax3(mx1, __uint_as_float(r2[i]), __uint_as_float(r3[i]));
+        }
+        const float mx = fmaxf(fmaf(mx0, p.scale_log2, b0), fmaf(mx1, p.scale_log2, b1));
         const float m_new = fmaxf(m_ref, mx);
         const bool grow = m_new > m_ref + RESCALE_THRESHOLD;   // also true on the first tile (m_ref = -inf)
         if (j > 0 && __any_sync(0xffffffffu, grow)) {
@@ -418,26 +451,27 @@ attn_tc_kernel(const __grid_constant__ AttnParams p, const __grid_constant__ Map
           l_sum *= f;
         }
         if (grow) m_ref = m_new;
-        // pass 2: p = exp2(logit - m_ref), row sum in fp32, P as bf16 pairs into the S columns
-#pragma unroll
-        for (int c = 0; c < 4; ++c) {
-          uint32_t r[32];
-          tmem_ld32(t_s + c * 32, r);
-          tmem_wait_ld();
-          const int nv = (c < 2 ? s0.n_valid : s1.n_valid) - (c & 1) * 32;
-          const float bb = (c < 2 ? b0 : b1) - m_ref;
+        // p = exp2(logit - m_ref); row sum in fp32; P as bf16 pairs into the columns S occupied
+        // (keys 32c..32c+31 -> P columns 16c..16c+15; the whole row of S is already in registers)
+        const float bb0 = b0 - m_ref, bb1 = b1 - m_ref;
+        float sum_a = 0.f, sum_b = 0.f;
+        auto exp_chunk = [&](const uint32_t (&rc)[32], float bb, int c) {
           uint32_t pk[16];
 #pragma unroll
           for (int i = 0; i < 32; i += 2) {
-            float e0 = i < nv ? exp2f(fmaf(__uint_as_float(r[i]), p.scale_log2, bb)) : 0.f;
-            float e1 = i + 1 < nv ? exp2f(fmaf(__uint_as_float(r[i + 1]), p.scale_log2, bb)) : 0.f;
-            l_sum += e0 + e1;
+            float e0 = ex2_approx(fmaf(__uint_as_float(rc[i]), p.scale_log2, bb));
+            float e1 = ex2_approx(fmaf(__uint_as_float(rc[i + 1]), p.scale_log2, bb));
+            sum_a += e0;
+            sum_b += e1;
             pk[i >> 1] = pack_bf16(e0, e1);
           }
-          // chunk c covers keys 32c..32c+31 -> P columns 16c..16c+15.  Column 16c+15 <= 32c+31 has
-          // been read already for every c, so writing never clobbers unread logits.
           tmem_st16(t_s + c * 16, pk);
-        }
+        };
+        exp_chunk(r0, bb0, 0);
+        exp_chunk(r1, bb0, 1);
+        exp_chunk(r2, bb1, 2);
+        exp_chunk(r3, bb1, 3);
+        l_sum += sum_a + sum_b;
         tmem_wait_st();
         tc_fence_before();
         mbar_arrive(bar(P_FULL + x));
