@@ -95,7 +95,7 @@ def exported_symbols():
 def _load() -> C.CDLL:
     path = lib_path()
     if not os.path.exists(path):
-        raise ImportError(f"{path} is missing: build it with `python -m paper_2605_14877_b200.build` "
+        raise ImportError(f"{path} is missing: build it with `python paper_2605_14877_b200/build.py` "
                           "(the CUDA library is the only implementation; there is no fallback)")
     return C.CDLL(path)
 
