@@ -179,6 +179,7 @@ def main():
     ap.add_argument("--layout", default="paged", choices=["paged", "ragged"])
     ap.add_argument("--kernel", default="auto", choices=["auto", "generic", "tcgen05"])
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-e2e", action="store_true", help="skip the host-buffer leg (profiling runs)")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
 
@@ -302,16 +303,18 @@ def main():
         for i in ids:
             hk.heatkv_seq_close(ses.ctx, i)
 
-    sweep_e2e()
-    barrier()
-    t0 = time.perf_counter()
-    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-    e0.record(stream)
-    for _ in range(e2e_steps):
+    e2e_ms = float("nan")
+    if not args.no_e2e:
         sweep_e2e()
-    e1.record(stream)
-    barrier()
-    e2e_ms = max(e0.elapsed_time(e1), 1e3 * (time.perf_counter() - t0)) / e2e_steps
+        barrier()
+        t0 = time.perf_counter()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record(stream)
+        for _ in range(e2e_steps):
+            sweep_e2e()
+        e1.record(stream)
+        barrier()
+        e2e_ms = max(e0.elapsed_time(e1), 1e3 * (time.perf_counter() - t0)) / e2e_steps
     h2d = 3 * q.numel() * 2
     d2h = q.numel() * 2
 

@@ -48,15 +48,16 @@ enum Bar : uint32_t {
   K_FULL = 2, K_EMPTY = 4,      // +stage
   V_FULL = 6, V_EMPTY = 8,      // +stage
   S_FULL = 10,                  // +x  S_x of tile j is in TMEM
-  P_FULL = 12,                  // +x  P_x of tile j is in TMEM (128 arrivals)
-  PV_DONE = 14,                 // +x  O_x includes tile j
-  N_BARS = 16
+  P_FULL = 12,                  // +2x+h  half h (keys 64h..64h+63) of P_x of tile j is in TMEM (128 arrivals)
+  PV_DONE = 16,                 // +x  O_x includes tile j
+  N_BARS = 18
 };
 constexpr uint32_t SM_TMEM_PTR = SM_BAR + N_BARS * 8;
 constexpr uint32_t SM_ABORT = SM_TMEM_PTR + 4;
 
-constexpr uint32_t WAIT_LIMIT = 1u << 20;               // about a second with the hint below
+constexpr uint32_t WAIT_LIMIT = 1u << 22;               // tries per wait; each try blocks for a bounded time
 constexpr float RESCALE_THRESHOLD = 8.0f;               // log2 units
+constexpr int POLY_PHASE = 3;                           // which pair of every four takes the polynomial exp2
 
 __device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
   asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count));
@@ -71,10 +72,10 @@ __device__ __forceinline__ bool mbar_try(uint32_t bar, uint32_t parity) {
   uint32_t ok;
   asm volatile(
       "{\n\t.reg .pred p;\n\t"
-      "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2, %3;\n\t"
+      "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
       "selp.u32 %0, 1, 0, p;\n\t}"
       : "=r"(ok)
-      : "r"(bar), "r"(parity), "r"(1000u)            // suspend-time hint: about a microsecond per try
+      : "r"(bar), "r"(parity)
       : "memory");
   return ok != 0;
 }
@@ -166,6 +167,62 @@ __device__ __forceinline__ float ex2_approx(float x) {
   asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
   return y;
 }
+// ---- packed fp32 pairs (one issue slot for two lanes of work)
+__device__ __forceinline__ uint64_t pack2(float lo, float hi) {
+  uint64_t r;
+  asm("mov.b64 %0, {%1, %2};" : "=l"(r) : "f"(lo), "f"(hi));
+  return r;
+}
+__device__ __forceinline__ void unpack2(uint64_t v, float& lo, float& hi) {
+  asm("mov.b64 {%0, %1}, %2;" : "=f"(lo), "=f"(hi) : "l"(v));
+}
+__device__ __forceinline__ uint64_t fma2(uint64_t a, uint64_t b, uint64_t c) {
+  uint64_t d;
+  asm("fma.rn.f32x2 %0, %1, %2, %3;" : "=l"(d) : "l"(a), "l"(b), "l"(c));
+  return d;
+}
+__device__ __forceinline__ uint64_t add2(uint64_t a, uint64_t b) {
+  uint64_t d;
+  asm("add.rn.f32x2 %0, %1, %2;" : "=l"(d) : "l"(a), "l"(b));
+  return d;
+}
+__device__ __forceinline__ uint64_t sub2(uint64_t a, uint64_t b) {
+  uint64_t d;
+  asm("sub.rn.f32x2 %0, %1, %2;" : "=l"(d) : "l"(a), "l"(b));
+  return d;
+}
+// 2^x for a pair on the FMA pipe: x = n + f with n = round(x), f in [-1/2, 1/2]; a cubic fitted to
+// 2^f (relative error 7.5e-5, far below the bf16 step of P) gets n added to its exponent field.
+// x is clamped at -125 so the exponent stays in range (masked keys arrive as -inf and give 2^-125).
+__device__ __forceinline__ void exp2_poly2(uint64_t x, float& e0, float& e1) {
+  constexpr float MAGIC = 12582912.f;                  // 1.5 * 2^23: the sum's low mantissa bits hold round(x)
+  float x0, x1;
+  unpack2(x, x0, x1);
+  x0 = fmaxf(x0, -125.f);
+  x1 = fmaxf(x1, -125.f);
+  const uint64_t xc = pack2(x0, x1);
+  const uint64_t magic = pack2(MAGIC, MAGIC);
+  const uint64_t t = add2(xc, magic);
+  const uint64_t f = sub2(xc, sub2(t, magic));
+  uint64_t q = fma2(pack2(0.0551716685f, 0.0551716685f), f, pack2(0.242611125f, 0.242611125f));
+  q = fma2(q, f, pack2(0.693260968f, 0.693260968f));
+  q = fma2(q, f, pack2(0.999928057f, 0.999928057f));
+  float t0, t1, q0, q1;
+  unpack2(t, t0, t1);
+  unpack2(q, q0, q1);
+  e0 = __uint_as_float(__float_as_uint(q0) + (__float_as_uint(t0) << 23));
+  e1 = __uint_as_float(__float_as_uint(q1) + (__float_as_uint(t1) << 23));
+}
+// One lane of a converged warp.  Role loops run on all 32 lanes (uniform control flow, descriptors in
+// uniform registers); only the asynchronous instruction itself is issued by the elected lane.
+__device__ __forceinline__ bool elect_one() {
+  uint32_t pred;
+  asm volatile("{\n\t.reg .pred P;\n\telect.sync _|P, 0xffffffff;\n\tselp.u32 %0, 1, 0, P;\n\t}" : "=r"(pred));
+  return pred != 0;
+}
+__device__ __forceinline__ bool warp_wait(uint32_t bar, uint32_t parity, volatile uint32_t* abort_flag, uint32_t* status) {
+  return __all_sync(0xffffffffu, mbar_wait(bar, parity, abort_flag, status));
+}
 template <uint32_t N>
 __device__ __forceinline__ void reg_alloc() {
   asm volatile("setmaxnreg.inc.sync.aligned.u32 %0;" ::"n"(N));
@@ -229,7 +286,8 @@ attn_tc_kernel(const __grid_constant__ AttnParams p, const __grid_constant__ Map
   volatile uint32_t* tmem_ptr_smem = reinterpret_cast<volatile uint32_t*>(sgen + SM_TMEM_PTR);
   auto bar = [&](uint32_t which) { return sbase + SM_BAR + which * 8; };
 
-  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  // the shuffle makes the warp index provably warp-uniform, so role code stays on the uniform datapath
+  const int warp = __shfl_sync(0xffffffffu, (int)(threadIdx.x >> 5), 0), lane = threadIdx.x & 31;
   const int seq = blockIdx.z;
   const int q0 = blockIdx.x * (2 * BM);
   const int nq = (q0 + BM < p.t_q) ? 2 : 1;          // does tile B hold any query?
@@ -255,7 +313,8 @@ attn_tc_kernel(const __grid_constant__ AttnParams p, const __grid_constant__ Map
     }
     for (int x = 0; x < 2; ++x) {
       mbar_init(bar(S_FULL + x), 1);
-      mbar_init(bar(P_FULL + x), BM);
+      mbar_init(bar(P_FULL + 2 * x), BM);
+      mbar_init(bar(P_FULL + 2 * x + 1), BM);
       mbar_init(bar(PV_DONE + x), 1);
     }
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
@@ -277,15 +336,18 @@ attn_tc_kernel(const __grid_constant__ AttnParams p, const __grid_constant__ Map
     reg_dealloc<72>();
   if (warp == 0) {
     // ------------------------------------------------------------------ TMA producer
-    if (lane == 0) {
+    {
+      const bool leader = elect_one();
       uint32_t armed_k = 0, armed_v = 0;               // stage -> a copy was issued at least once
       uint32_t par_k[KV_STAGES] = {0, 0}, par_v[KV_STAGES] = {0, 0};
-      for (int x = 0; x < nq; ++x) {
-        mbar_expect_tx(bar(Q_FULL + x), TILE_BYTES);
-        for (int ch = 0; ch < 2; ++ch)
-          for (int hf = 0; hf < 2; ++hf)
-            tma_load_4d(sbase + SM_Q + x * TILE_BYTES + ch * HALF_COLS_BYTES + hf * SLOT_BYTES, &maps.q, ch * 64,
-                        q0 + x * BM + hf * HALF, head, seq, bar(Q_FULL + x));
+      if (leader) {
+        for (int x = 0; x < nq; ++x) {
+          mbar_expect_tx(bar(Q_FULL + x), TILE_BYTES);
+          for (int ch = 0; ch < 2; ++ch)
+            for (int hf = 0; hf < 2; ++hf)
+              tma_load_4d(sbase + SM_Q + x * TILE_BYTES + ch * HALF_COLS_BYTES + hf * SLOT_BYTES, &maps.q, ch * 64,
+                          q0 + x * BM + hf * HALF, head, seq, bar(Q_FULL + x));
+        }
       }
       bool ok = true;
       for (int j = 0; j < n_tiles && ok; ++j) {
@@ -294,31 +356,36 @@ attn_tc_kernel(const __grid_constant__ AttnParams p, const __grid_constant__ Map
         Slot sl[2];
         for (int hf = 0; hf < 2; ++hf) sl[hf] = get_slot(2 * j + hf, descs, n_desc, n_slots, base_row, p.n_own, p.step);
         // K first: the S product of the next tile needs it earliest
-        if (use > 0) ok = mbar_wait(bar(K_EMPTY + st), (use - 1) & 1, abort_flag, p.status);
+        if (use > 0) ok = warp_wait(bar(K_EMPTY + st), (use - 1) & 1, abort_flag, p.status);
         if (!ok) break;
-        mbar_expect_tx(bar(K_FULL + st), TILE_BYTES);
         armed_k |= 1u << st;
         par_k[st] = use & 1;
-        for (int hf = 0; hf < 2; ++hf)
-          for (int ch = 0; ch < 2; ++ch) {
-            uint32_t dst = sbase + SM_K + st * TILE_BYTES + ch * HALF_COLS_BYTES + hf * SLOT_BYTES;
-            if (sl[hf].pool_row >= 0) tma_load_2d(dst, &maps.k_pool, ch * 64, sl[hf].pool_row, bar(K_FULL + st));
-            else tma_load_4d(dst, &maps.k_own, ch * 64, -sl[hf].pool_row - 1, head, seq, bar(K_FULL + st));
-          }
-        if (use > 0) ok = mbar_wait(bar(V_EMPTY + st), (use - 1) & 1, abort_flag, p.status);
+        if (leader) {
+          mbar_expect_tx(bar(K_FULL + st), TILE_BYTES);
+          for (int hf = 0; hf < 2; ++hf)
+            for (int ch = 0; ch < 2; ++ch) {
+              uint32_t dst = sbase + SM_K + st * TILE_BYTES + ch * HALF_COLS_BYTES + hf * SLOT_BYTES;
+              if (sl[hf].pool_row >= 0) tma_load_2d(dst, &maps.k_pool, ch * 64, sl[hf].pool_row, bar(K_FULL + st));
+              else tma_load_4d(dst, &maps.k_own, ch * 64, -sl[hf].pool_row - 1, head, seq, bar(K_FULL + st));
+            }
+        }
+        if (use > 0) ok = warp_wait(bar(V_EMPTY + st), (use - 1) & 1, abort_flag, p.status);
         if (!ok) break;
-        mbar_expect_tx(bar(V_FULL + st), TILE_BYTES);
         armed_v |= 1u << st;
         par_v[st] = use & 1;
-        for (int hf = 0; hf < 2; ++hf)
-          for (int ch = 0; ch < 2; ++ch) {
-            uint32_t dst = sbase + SM_V + st * TILE_BYTES + ch * HALF_COLS_BYTES + hf * SLOT_BYTES;
-            if (sl[hf].pool_row >= 0) tma_load_2d(dst, &maps.v_pool, ch * 64, sl[hf].pool_row, bar(V_FULL + st));
-            else tma_load_4d(dst, &maps.v_own, ch * 64, -sl[hf].pool_row - 1, head, seq, bar(V_FULL + st));
-          }
+        if (leader) {
+          mbar_expect_tx(bar(V_FULL + st), TILE_BYTES);
+          for (int hf = 0; hf < 2; ++hf)
+            for (int ch = 0; ch < 2; ++ch) {
+              uint32_t dst = sbase + SM_V + st * TILE_BYTES + ch * HALF_COLS_BYTES + hf * SLOT_BYTES;
+              if (sl[hf].pool_row >= 0) tma_load_2d(dst, &maps.v_pool, ch * 64, sl[hf].pool_row, bar(V_FULL + st));
+              else tma_load_4d(dst, &maps.v_own, ch * 64, -sl[hf].pool_row - 1, head, seq, bar(V_FULL + st));
+            }
+        }
+        __syncwarp();
       }
       if (!ok) {
-        // leaving early: let every copy this thread started land before the CTA exits
+        // leaving early: let every copy this warp started land before the CTA exits
         for (int s = 0; s < KV_STAGES; ++s) {
           if (armed_k & (1u << s))
             for (uint32_t it = 0; it < WAIT_LIMIT && !mbar_try(bar(K_FULL + s), par_k[s]); ++it) {}
@@ -331,7 +398,8 @@ attn_tc_kernel(const __grid_constant__ AttnParams p, const __grid_constant__ Map
     }
   } else if (warp == 1) {
     // ------------------------------------------------------------------ MMA issuer
-    if (lane == 0) {
+    {
+      const bool leader = elect_one();
       constexpr uint32_t IDESC_S = instr_desc(BM, BN, 0, 0);     // Q, K both K-major
       constexpr uint32_t IDESC_PV = instr_desc(BM, D, 0, 1);     // P from TMEM, V MN-major
       bool ok = true;
@@ -343,44 +411,57 @@ attn_tc_kernel(const __grid_constant__ AttnParams p, const __grid_constant__ Map
           mma_ss(tmem + x * 128, smem_desc(qa + off, 16, 1024), smem_desc(ka + off, 16, 1024), IDESC_S, ks > 0);
         }
       };
-      auto issue_pv = [&](int x, int st, bool first) {
+      // keys 64h .. 64h+63 of the tile: four K=16 steps
+      auto issue_pv = [&](int x, int st, int h, bool first) {
         const uint32_t va = sbase + SM_V + st * TILE_BYTES;
 #pragma unroll
-        for (int ks = 0; ks < BN / 16; ++ks)
+        for (int ks = 4 * h; ks < 4 * h + 4; ++ks)
           mma_ts(tmem + 256 + x * 128, tmem + x * 128 + ks * 8, smem_desc(va + ks * 2048, HALF_COLS_BYTES, 1024),
                  IDESC_PV, !(first && ks == 0));
       };
-      for (int x = 0; x < nq && ok; ++x) ok = mbar_wait(bar(Q_FULL + x), 0, abort_flag, p.status);
-      if (ok) ok = mbar_wait(bar(K_FULL + 0), 0, abort_flag, p.status);
+      for (int x = 0; x < nq && ok; ++x) ok = warp_wait(bar(Q_FULL + x), 0, abort_flag, p.status);
+      if (ok) ok = warp_wait(bar(K_FULL + 0), 0, abort_flag, p.status);
       if (ok) {
         tc_fence_after();
-        for (int x = 0; x < nq; ++x) {
-          issue_s(x, 0);
-          tc_commit(bar(S_FULL + x));
+        if (leader) {
+          for (int x = 0; x < nq; ++x) {
+            issue_s(x, 0);
+            tc_commit(bar(S_FULL + x));
+          }
+          tc_commit(bar(K_EMPTY + 0));
         }
-        tc_commit(bar(K_EMPTY + 0));
+        __syncwarp();
       }
       for (int j = 0; j < n_tiles && ok; ++j) {
         const int st = j % KV_STAGES, stn = (j + 1) % KV_STAGES;
         const uint32_t par = (uint32_t)(j / KV_STAGES) & 1, parn = (uint32_t)((j + 1) / KV_STAGES) & 1;
         const bool more = j + 1 < n_tiles;
-        ok = mbar_wait(bar(V_FULL + st), par, abort_flag, p.status);
-        if (ok && more) ok = mbar_wait(bar(K_FULL + stn), parn, abort_flag, p.status);
+        ok = warp_wait(bar(V_FULL + st), par, abort_flag, p.status);
+        if (ok && more) ok = warp_wait(bar(K_FULL + stn), parn, abort_flag, p.status);
         for (int x = 0; x < nq && ok; ++x) {
-          ok = mbar_wait(bar(P_FULL + x), j & 1, abort_flag, p.status);
+          ok = warp_wait(bar(P_FULL + 2 * x), j & 1, abort_flag, p.status);
           if (!ok) break;
           tc_fence_after();
-          issue_pv(x, st, j == 0);
-          tc_commit(bar(PV_DONE + x));
-          if (more) {
-            issue_s(x, stn);
-            tc_commit(bar(S_FULL + x));
+          if (leader) issue_pv(x, st, 0, j == 0);
+          __syncwarp();
+          ok = warp_wait(bar(P_FULL + 2 * x + 1), j & 1, abort_flag, p.status);
+          if (!ok) break;
+          tc_fence_after();
+          if (leader) {
+            issue_pv(x, st, 1, false);
+            tc_commit(bar(PV_DONE + x));
+            if (more) {
+              issue_s(x, stn);
+              tc_commit(bar(S_FULL + x));
+            }
           }
+          __syncwarp();
         }
-        if (ok) {
+        if (ok && leader) {
           tc_commit(bar(V_EMPTY + st));
           if (more) tc_commit(bar(K_EMPTY + stn));
         }
+        __syncwarp();
       }
     }
   }
@@ -422,13 +503,23 @@ attn_tc_kernel(const __grid_constant__ AttnParams p, const __grid_constant__ Map
           }
         }
         // row maximum: the logit is raw * scale + bias(half) with scale > 0, so take the raw maxima
-        float mx0 = fmaxf(__uint_as_float(r0[0]), __uint_as_float(r1[0]));
-        float mx1 = fmaxf(__uint_as_float(r2[0]), __uint_as_float(r3[0]));
+        // (eight independent chains keep the dependent depth short)
+        float mq[8];
 #pragma unroll
-        for (int i = 1; i < 32; ++i) {
-          mx0 = fmax3(mx0, __uint_as_float(r0[i]), __uint_as_float(r1[i]));
-          mx1 = fmax3(mx1, __uint_as_float(r2[i]), __uint_as_float(r3[i]));
+        for (int c = 0; c < 4; ++c) {
+          mq[c] = fmaxf(__uint_as_float(r0[c]), __uint_as_float(r1[c]));
+          mq[4 + c] = fmaxf(__uint_as_float(r2[c]), __uint_as_float(r3[c]));
         }
+#pragma unroll
+        for (int i = 4; i < 32; i += 4) {
+#pragma unroll
+          for (int c = 0; c < 4; ++c) {
+            mq[c] = fmax3(mq[c], __uint_as_float(r0[i + c]), __uint_as_float(r1[i + c]));
+            mq[4 + c] = fmax3(mq[4 + c], __uint_as_float(r2[i + c]), __uint_as_float(r3[i + c]));
+          }
+        }
+        const float mx0 = fmaxf(fmaxf(mq[0], mq[1]), fmaxf(mq[2], mq[3]));
+        const float mx1 = fmaxf(fmaxf(mq[4], mq[5]), fmaxf(mq[6], mq[7]));
         const float mx = fmaxf(fmaf(mx0, p.scale_log2, b0), fmaf(mx1, p.scale_log2, b1));
         const float m_new = fmaxf(m_ref, mx);
         const bool grow = m_new > m_ref + RESCALE_THRESHOLD;   // also true on the first tile (m_ref = -inf)
@@ -452,29 +543,45 @@ attn_tc_kernel(const __grid_constant__ AttnParams p, const __grid_constant__ Map
         }
         if (grow) m_ref = m_new;
         // p = exp2(logit - m_ref); row sum in fp32; P as bf16 pairs into the columns S occupied
-        // (keys 32c..32c+31 -> P columns 16c..16c+15; the whole row of S is already in registers)
-        const float bb0 = b0 - m_ref, bb1 = b1 - m_ref;
-        float sum_a = 0.f, sum_b = 0.f;
-        auto exp_chunk = [&](const uint32_t (&rc)[32], float bb, int c) {
+        // (keys 32c..32c+31 -> P columns 16c..16c+15; the whole row of S is already in registers).
+        // One pair in four takes the polynomial on the FMA pipe, the rest the MUFU unit: the tile's
+        // 16 384 exponentials would otherwise keep MUFU busy as long as the tensor pipe needs for
+        // the tile's two products.
+        const uint64_t scale2 = pack2(p.scale_log2, p.scale_log2);
+        uint64_t sum2 = pack2(0.f, 0.f);
+        auto exp_chunk = [&](const uint32_t (&rc)[32], uint64_t bb2, int c) {
           uint32_t pk[16];
 #pragma unroll
           for (int i = 0; i < 32; i += 2) {
-            float e0 = ex2_approx(fmaf(__uint_as_float(rc[i]), p.scale_log2, bb));
-            float e1 = ex2_approx(fmaf(__uint_as_float(rc[i + 1]), p.scale_log2, bb));
-            sum_a += e0;
-            sum_b += e1;
+            const uint64_t xx = fma2(pack2(__uint_as_float(rc[i]), __uint_as_float(rc[i + 1])), scale2, bb2);
+            float e0, e1;
+            if (((i >> 1) & 3) == POLY_PHASE) {
+              exp2_poly2(xx, e0, e1);
+            } else {
+              float x0, x1;
+              unpack2(xx, x0, x1);
+              e0 = ex2_approx(x0);
+              e1 = ex2_approx(x1);
+            }
+            sum2 = add2(sum2, pack2(e0, e1));
             pk[i >> 1] = pack_bf16(e0, e1);
           }
           tmem_st16(t_s + c * 16, pk);
         };
+        const uint64_t bb0 = pack2(b0 - m_ref, b0 - m_ref), bb1 = pack2(b1 - m_ref, b1 - m_ref);
         exp_chunk(r0, bb0, 0);
         exp_chunk(r1, bb0, 1);
-        exp_chunk(r2, bb1, 2);
-        exp_chunk(r3, bb1, 3);
-        l_sum += sum_a + sum_b;
         tmem_wait_st();
         tc_fence_before();
-        mbar_arrive(bar(P_FULL + x));
+        mbar_arrive(bar(P_FULL + 2 * x));                      // the PV product of keys 0..63 may start
+        exp_chunk(r2, bb1, 2);
+        exp_chunk(r3, bb1, 3);
+        float sa, sb;
+        unpack2(sum2, sa, sb);
+        l_sum += sa + sb;
+        tmem_wait_st();
+        tc_fence_before();
+        mbar_arrive(bar(P_FULL + 2 * x + 1));
       }
       if (ok) ok = __all_sync(0xffffffffu, mbar_wait(bar(PV_DONE + x), (n_tiles - 1) & 1, abort_flag, p.status));
       if (ok) {
