@@ -66,7 +66,7 @@ class ClockSampler:
             if probe.returncode != 0 or "not a valid" in (probe.stdout + probe.stderr).lower():
                 query = self.Q_OLD
             self.proc = subprocess.Popen(["nvidia-smi", f"--id={self.index}", f"--query-gpu={query}",
-                                          "--format=csv,noheader,nounits", "-lms", "100"],
+                                          "--format=csv,noheader,nounits", "-lms", "50"],
                                          stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
             self.thread = threading.Thread(target=self._read, daemon=True)
             self.thread.start()
@@ -173,7 +173,7 @@ def run_reference(args, rank):
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=20)
+    ap.add_argument("--steps", type=int, default=300)
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--layout", default="paged", choices=["paged", "ragged"])

@@ -432,12 +432,14 @@ attn_tc_kernel(const __grid_constant__ AttnParams p, const __grid_constant__ Map
         }
         __syncwarp();
       }
+      // Waits for K and V sit where the tensor pipe still has queued work: the next tile's V at the end
+      // of an iteration, the next tile's K between PV_A and S_A.  The hand-over of P is then the only
+      // wait between the last S product of one tile and the first PV product of the next.
+      if (ok) ok = warp_wait(bar(V_FULL + 0), 0, abort_flag, p.status);
       for (int j = 0; j < n_tiles && ok; ++j) {
         const int st = j % KV_STAGES, stn = (j + 1) % KV_STAGES;
-        const uint32_t par = (uint32_t)(j / KV_STAGES) & 1, parn = (uint32_t)((j + 1) / KV_STAGES) & 1;
+        const uint32_t parn = (uint32_t)((j + 1) / KV_STAGES) & 1;
         const bool more = j + 1 < n_tiles;
-        ok = warp_wait(bar(V_FULL + st), par, abort_flag, p.status);
-        if (ok && more) ok = warp_wait(bar(K_FULL + stn), parn, abort_flag, p.status);
         for (int x = 0; x < nq && ok; ++x) {
           ok = warp_wait(bar(P_FULL + 2 * x), j & 1, abort_flag, p.status);
           if (!ok) break;
@@ -450,18 +452,24 @@ attn_tc_kernel(const __grid_constant__ AttnParams p, const __grid_constant__ Map
           if (leader) {
             issue_pv(x, st, 1, false);
             tc_commit(bar(PV_DONE + x));
-            if (more) {
+          }
+          __syncwarp();
+          if (more) {
+            if (x == 0) ok = warp_wait(bar(K_FULL + stn), parn, abort_flag, p.status);
+            if (!ok) break;
+            if (leader) {
               issue_s(x, stn);
               tc_commit(bar(S_FULL + x));
             }
+            __syncwarp();
           }
-          __syncwarp();
         }
         if (ok && leader) {
           tc_commit(bar(V_EMPTY + st));
           if (more) tc_commit(bar(K_EMPTY + stn));
         }
         __syncwarp();
+        if (ok && more) ok = warp_wait(bar(V_FULL + stn), parn, abort_flag, p.status);
       }
     }
   }
