@@ -55,9 +55,11 @@ __global__ void __launch_bounds__(GTHREADS, 2) attn_generic_kernel(const __grid_
   using SM = GenericSmem<D>;
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   const int g = lane >> 2, qd = lane & 3;
-  const int seq = blockIdx.z;
+  // attention: grid = (query tiles, sequences, heads by descending key count), so the heaviest heads of
+  // every sequence are dispatched first; calibration: grid = (query tiles, heads, sequences)
+  const int seq = CALIB ? blockIdx.z : blockIdx.y;
   const int q0 = blockIdx.x * GM;
-  int head = blockIdx.y;
+  int head = CALIB ? blockIdx.y : blockIdx.z;
 
   const int2* descs = nullptr;
   int n_desc = 0;
@@ -65,7 +67,7 @@ __global__ void __launch_bounds__(GTHREADS, 2) attn_generic_kernel(const __grid_
   if (!CALIB) {
     PlanView pv(p.seqs[seq].plan);
     const int u = (p.step * p.L + p.layer) * p.H;
-    head = pv.order()[u + blockIdx.y];                   // heavy heads first
+    head = pv.order()[u + blockIdx.z];                   // heavy heads first
     descs = pv.descs() + pv.attn_begin()[u + head];
     n_desc = pv.attn_cnt()[u + head];
     base_row = p.seqs[seq].base_row;
@@ -343,7 +345,7 @@ static cudaError_t launch_one(const AttnParams& p, int n_seq, cudaStream_t strea
     if (e != cudaSuccess) return e;
     configured = true;
   }
-  dim3 grid((p.t_q + GM - 1) / GM, p.H, n_seq);
+  dim3 grid((p.t_q + GM - 1) / GM, CALIB ? p.H : n_seq, CALIB ? n_seq : p.H);
   kern<<<grid, GTHREADS, GenericSmem<D>::BYTES, stream>>>(p);
   return cudaGetLastError();
 }

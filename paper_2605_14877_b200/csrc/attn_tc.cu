@@ -55,9 +55,9 @@ enum Bar : uint32_t {
 constexpr uint32_t SM_TMEM_PTR = SM_BAR + N_BARS * 8;
 constexpr uint32_t SM_ABORT = SM_TMEM_PTR + 4;
 
-constexpr uint32_t WAIT_LIMIT = 1u << 22;               // tries per wait; each try blocks for a bounded time
+constexpr uint32_t WAIT_LIMIT = 1u << 18;               // tries per wait; each try blocks for a bounded time
 constexpr float RESCALE_THRESHOLD = 8.0f;               // log2 units
-constexpr int POLY_PHASE = 3;                           // which pair of every four takes the polynomial exp2
+constexpr int POLY_MASK = 3;                            // pairs whose index has these bits set take the polynomial exp2 (3: one pair in four)
 
 __device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
   asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count));
@@ -288,13 +288,15 @@ attn_tc_kernel(const __grid_constant__ AttnParams p, const __grid_constant__ Map
 
   // the shuffle makes the warp index provably warp-uniform, so role code stays on the uniform datapath
   const int warp = __shfl_sync(0xffffffffu, (int)(threadIdx.x >> 5), 0), lane = threadIdx.x & 31;
-  const int seq = blockIdx.z;
+  // grid = (query tile pairs, sequences, heads by descending key count): the heaviest heads of every
+  // sequence are dispatched first
+  const int seq = blockIdx.y;
   const int q0 = blockIdx.x * (2 * BM);
   const int nq = (q0 + BM < p.t_q) ? 2 : 1;          // does tile B hold any query?
 
   PlanView pv(p.seqs[seq].plan);
   const int u = (p.step * p.L + p.layer) * p.H;
-  const int head = pv.order()[u + blockIdx.y];
+  const int head = pv.order()[u + blockIdx.z];
   const int2* descs = pv.descs() + pv.attn_begin()[u + head];
   const int n_desc = pv.attn_cnt()[u + head];
   const int64_t base_row = p.seqs[seq].base_row;
@@ -302,7 +304,7 @@ attn_tc_kernel(const __grid_constant__ AttnParams p, const __grid_constant__ Map
   const int n_tiles = (n_slots + 1) / 2;
 
   if (threadIdx.x == 0) {
-    *abort_flag = 0;
+    *abort_flag = *reinterpret_cast<volatile uint32_t*>(p.status) != 0;   // an earlier CTA gave up: do not wait again
     mbar_init(bar(Q_FULL + 0), 1);
     mbar_init(bar(Q_FULL + 1), 1);
     for (int s = 0; s < KV_STAGES; ++s) {
@@ -563,7 +565,7 @@ attn_tc_kernel(const __grid_constant__ AttnParams p, const __grid_constant__ Map
           for (int i = 0; i < 32; i += 2) {
             const uint64_t xx = fma2(pack2(__uint_as_float(rc[i]), __uint_as_float(rc[i + 1])), scale2, bb2);
             float e0, e1;
-            if (((i >> 1) & 3) == POLY_PHASE) {
+            if (((i >> 1) & POLY_MASK) == POLY_MASK) {
               exp2_poly2(xx, e0, e1);
             } else {
               float x0, x1;
@@ -709,7 +711,7 @@ cudaError_t launch_attn_tc(TcState* st, const AttnParams& p, int d, int n_seq, b
       !encode_4d(st, &maps.k_own, p.k_new, p.n_own, p.H, n_seq, p.kv_tok, p.kv_head, p.kv_seq) ||
       !encode_4d(st, &maps.v_own, p.v_new, p.n_own, p.H, n_seq, p.kv_tok, p.kv_head, p.kv_seq))
     return cudaErrorInvalidValue;
-  dim3 grid((p.t_q + 2 * tc::BM - 1) / (2 * tc::BM), p.H, n_seq);
+  dim3 grid((p.t_q + 2 * tc::BM - 1) / (2 * tc::BM), n_seq, p.H);
   tc::attn_tc_kernel<<<grid, tc::THREADS, tc::SM_ALLOC, stream>>>(p, maps);
   *launches = 1;
   return cudaGetLastError();
