@@ -38,6 +38,9 @@ CALIB_SEEDS = (100, 101, 102, 103)
 DATA_SEED = 0
 METRIC = "images_per_sec_scale_step_attention_2b_single_layer_20x"
 UNIT = "images/s"
+# dram__bytes_read.sum + dram__bytes_write.sum of the dominant kernel's launches of one sweep, from the ncu
+# capture summarised under profiles/; None once the kernel changed after the capture
+TRAFFIC_BYTES_PER_SWEEP = None
 
 
 def peaks():
@@ -118,50 +121,75 @@ def attention_flops(shape, am, n_seq):
     return out
 
 
-def oracle_unit_seconds(shape, n_units, bias):
-    """Times the CPU oracle (attention of all 13 steps + cache contents) on `n_units`
-    (seq, head) pairs of the workload.  Returns (seconds, threads)."""
+def oracle_context(shape):
+    """Inputs of the oracle timing: the oracle's own schedule from seeded scores, one sequence of
+    the workload widened to fp64."""
     from oracle import heatkv_oracle as O
     scores = W.synthetic_scas(shape, 0)
     sch = O.heatkv_schedule(scores, B_BUDGET, shape.s, shape.sides)
     q, k, v = W.qkv_layer(shape, DATA_SEED, 0, n_seq=1)
     f = lambda x: O.bf16_bits_to_f64(W.bf16_bits(x))
-    qh, kh, vh = f(q), f(k), f(v)
-    kb, vb = W.bf16_bits(k), W.bf16_bits(v)
-    sm = 1.0 / math.sqrt(shape.d)
+    return {"O": O, "sch": sch, "q": f(q), "k": f(k), "v": f(v), "kb": W.bf16_bits(k), "vb": W.bf16_bits(v),
+            "bias": W.seg_bias_current_scale(shape, DATA_SEED), "sm": 1.0 / math.sqrt(shape.d)}
+
+
+def oracle_flops(shape, ctx, head, steps):
+    """Algorithmic attention flops (4*d*t_k*n_vis) of the given 1-based steps for one head under the
+    oracle's schedule."""
+    O, sch = ctx["O"], ctx["sch"]
+    tot = 0
+    for step in steps:
+        n_vis = sum(int(sch.t[i - 1]) for i in O.visible_scales(sch, step, 0, head)) + shape.t[step - 1]
+        tot += 4 * shape.d * shape.t[step - 1] * n_vis
+    return tot
+
+
+def oracle_seconds(shape, ctx, head, steps):
+    """Times the CPU oracle as it stands (attention + cache contents) on one (seq, head) unit for the
+    given 1-based steps."""
+    O, sch = ctx["O"], ctx["sch"]
     t0 = time.perf_counter()
-    for u in range(n_units):
-        h = u % shape.H
-        for step in range(1, shape.K + 1):
-            lo, hi = (shape.c[step - 2] if step > 1 else 0), shape.c[step - 1]
-            brow = bias[0, step - 1, h].astype(np.float64)
-            O.scale_attention(qh[0, h, lo:hi], kh[0, h], vh[0, h], sch, step, 0, h, sm, brow)
-            if step < shape.K:
-                O.cache_after_layer(kb[0, h], vb[0, h], sch, step, 0, h)
-    dt = time.perf_counter() - t0
-    return dt, torch.get_num_threads()
+    for step in steps:
+        lo, hi = (shape.c[step - 2] if step > 1 else 0), shape.c[step - 1]
+        brow = ctx["bias"][0, step - 1, head].astype(np.float64)
+        O.scale_attention(ctx["q"][0, head, lo:hi], ctx["k"][0, head], ctx["v"][0, head], sch, step, 0, head,
+                          ctx["sm"], brow)
+        if step < shape.K:
+            O.cache_after_layer(ctx["kb"][0, head], ctx["vb"][0, head], sch, step, 0, head)
+    return time.perf_counter() - t0
+
+
+def oracle_images_per_s(shape, ctx, samples):
+    """samples: list of (head, steps).  Extrapolates to one image (n_seq * H units, all scales) by
+    algorithmic flops.  Returns (images/s, seconds spent, flops covered / flops of one image)."""
+    all_steps = list(range(1, shape.K + 1))
+    image_flops = shape.n_seq * sum(oracle_flops(shape, ctx, h, all_steps) for h in range(shape.H))
+    secs = sum(oracle_seconds(shape, ctx, h, st) for h, st in samples)
+    done = sum(oracle_flops(shape, ctx, h, st) for h, st in samples)
+    return done / secs / image_flops, secs, done / image_flops
 
 
 def run_reference(args, rank):
-    """Reference arm: the CPU oracle as it stands, timed on the host cores."""
+    """Reference arm: the CPU oracle as it stands, timed on the host cores.  Every step times a
+    bounded sample (one (seq, head) unit, all scales or a rotating subset of them when K is large)
+    and the per-image rate is extrapolated by algorithmic flops."""
     if rank != 0:
         return
     shape = W.CFG2
-    bias = W.seg_bias_current_scale(shape, DATA_SEED)
-    units_per_step = 4
-    for _ in range(args.warmup):
-        oracle_unit_seconds(shape, 1, bias)
-    total = 0.0
-    threads = 1
-    for _ in range(args.steps):
-        dt, threads = oracle_unit_seconds(shape, units_per_step, bias)
-        total += dt
-    units_per_image = shape.n_seq * shape.H
-    sec_per_image = total / (args.steps * units_per_step) * units_per_image
-    value = 1.0 / sec_per_image
-    sample = f"{units_per_step} of {units_per_image} (seq, head) units per step, all 13 scales, extrapolated"
+    ctx = oracle_context(shape)
+    all_steps = list(range(1, shape.K + 1))
+    unit_s = oracle_seconds(shape, ctx, 0, all_steps)
+    for _ in range(max(args.warmup - 1, 0)):
+        oracle_seconds(shape, ctx, 0, all_steps[-2:])
+    budget_s = 150.0
+    stride = max(1, int(math.ceil(args.steps * unit_s / budget_s)))
+    samples = [(i % shape.H, [st for st in all_steps if (st + i) % stride == 0] or [shape.K]) for i in range(args.steps)]
+    value, secs, frac = oracle_images_per_s(shape, ctx, samples)
+    threads = torch.get_num_threads()
+    sample = (f"per step one (seq, head) unit of {shape.n_seq * shape.H}, every {stride}-th scale "
+              f"(all 13 when 1); {secs:.1f} s of CPU work = {frac:.3g} images, extrapolated by flops")
     line = {"impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus,
-            "steps": args.steps, "warmup": args.warmup, "ms_per_step": 1e3 * sec_per_image,
+            "steps": args.steps, "warmup": args.warmup, "ms_per_step": 1e3 / value,
             "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
             "config": {"workload": W.CFG2.name, "budget": B_BUDGET, "n_seq": shape.n_seq},
             "cpu_baseline": {"value": value, "unit": UNIT, "cores": threads, "kind": "oracle", "sample": sample},
@@ -178,6 +206,8 @@ def main():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--layout", default="paged", choices=["paged", "ragged"])
     ap.add_argument("--kernel", default="auto", choices=["auto", "generic", "tcgen05"])
+    ap.add_argument("--launch", default="graph", choices=["graph", "eager"],
+                    help="timed sweeps replay one captured CUDA graph of the 13-step sweep, or issue every call")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true", help="skip the host-buffer leg (profiling runs)")
     args = ap.parse_args()
@@ -206,7 +236,7 @@ def main():
     kernel = {"auto": hk.KERNEL_AUTO, "generic": hk.KERNEL_GENERIC, "tcgen05": hk.KERNEL_TCGEN05}[args.kernel]
     n_seq = shape.n_seq
     ses = Session(shape.L, shape.H, shape.d, shape.t, shape.s,
-                  pool_rows=n_seq * shape.L * shape.H * (shape.c[-2] + 64 * shape.K), layout=layout,
+                  pool_rows=2 * n_seq * shape.L * shape.H * (shape.c[-2] + 64 * shape.K), layout=layout,
                   kernel=kernel, device=str(dev))
     bias_np = W.seg_bias_current_scale(shape, DATA_SEED)
     bias = torch.from_numpy(bias_np).to(dev)
@@ -232,26 +262,31 @@ def main():
     am, km, nk, budget = hk.heatkv_schedule_masks(sch, shape.K, shape.L, shape.H)
     flops = attention_flops(shape, am, n_seq)
     calib_flops = sum(2 * shape.d * shape.t[k] * shape.c[k] for k in range(shape.K)) * shape.H * n_seq * len(CALIB_SEEDS)
+    tc_steps = [kk for kk in range(shape.K) if args.kernel != "generic" and (shape.t[kk] >= 256 or args.kernel == "tcgen05")]
 
-    # ---- device-resident inputs of the timed workload
+    # ---- device-resident inputs of the timed workload: one [n_seq, H, t_k, d] block per scale
     q, k, v = W.qkv_layer(shape, DATA_SEED, 0, device=dev)
-    out = torch.zeros_like(q)
+    qs_, ks_, vs_, os_ = [], [], [], []
+    for step in range(shape.K):
+        lo, hi = ses.step_slices(step)
+        qs_.append(q[:, :, lo:hi].contiguous()); ks_.append(k[:, :, lo:hi].contiguous())
+        vs_.append(v[:, :, lo:hi].contiguous()); os_.append(torch.zeros_like(qs_[-1]))
+    del q, k, v
     flush = torch.empty(256 << 20, dtype=torch.uint8, device=dev)
-    stream = torch.cuda.current_stream()
 
-    def sweep(events=None):
+    def sweep(events=None, bufs=None):
+        """One image pair through the layer: 13 x (pre-step eviction, attention, append/compaction)."""
+        stream = torch.cuda.current_stream()
+        bq, bk, bv, bo = bufs or (qs_, ks_, vs_, os_)
         ids = [hk.heatkv_seq_open(ses.ctx, sch) for _ in range(n_seq)]
         for step in range(shape.K):
             ses.pre_step(ids, step)
-            lo, hi = ses.step_slices(step)
-            qs, ks, vs, os_ = q[:, :, lo:hi], k[:, :, lo:hi], v[:, :, lo:hi], out[:, :, lo:hi]
-            st = hk.Strides.of(qs, ks, os_)
-            if events is not None:
+            if events is not None and step in events:
                 events[step][0].record(stream)
-            hk.heatkv_scale_attention(ses.ctx, ids, 0, step, qs, ks, vs, st, bias[0, step], os_)
-            if events is not None:
+            hk.heatkv_scale_attention(ses.ctx, ids, 0, step, bq[step], bk[step], bv[step], None, bias[0, step], bo[step])
+            if events is not None and step in events:
                 events[step][1].record(stream)
-            hk.heatkv_append_compact(ses.ctx, ids, 0, step, ks, vs, st)
+            hk.heatkv_append_compact(ses.ctx, ids, 0, step, bk[step], bv[step], None)
         for i in ids:
             hk.heatkv_seq_close(ses.ctx, i)
 
@@ -264,47 +299,77 @@ def main():
     for _ in range(args.warmup):
         sweep()
     barrier()
+    launches0 = hk.heatkv_launch_count(ses.ctx)
+    sweep()
+    launches_per_sweep = hk.heatkv_launch_count(ses.ctx) - launches0
+    graph = None
+    if args.launch == "graph":
+        # the calls are plain launches on the current stream once the schedule's plan is resident, so the
+        # whole sweep records into one graph; every replay issues the same kernels on the same buffers
+        side = torch.cuda.Stream()
+        side.wait_stream(torch.cuda.current_stream())
+        with torch.cuda.stream(side):
+            sweep()
+        torch.cuda.current_stream().wait_stream(side)
+        barrier()
+        graph = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(graph):
+            sweep()
+        for _ in range(args.warmup):
+            graph.replay()
+        barrier()
 
+    # ---- timed region: exactly K sweeps, L2 flushed (untimed) before each
+    stream = torch.cuda.current_stream()
     sampler = ClockSampler(local)
     sampler.start()
-    launches0 = hk.heatkv_launch_count(ses.ctx)
     step_events = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True))
                    for _ in range(args.steps)]
-    kern_events = [[(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True))
-                    for _ in range(shape.K)] for _ in range(args.steps)]
     barrier()
     for it in range(args.steps):
-        flush.fill_(it & 0xff)                         # evict L2 between timed steps (untimed)
+        flush.fill_(it & 0xff)
         step_events[it][0].record(stream)
-        sweep(kern_events[it])
+        if graph is not None:
+            graph.replay()
+        else:
+            sweep()
         step_events[it][1].record(stream)
     barrier()
-    launches = hk.heatkv_launch_count(ses.ctx) - launches0
     total_ms = sum(a.elapsed_time(b) for a, b in step_events)
-    per_step_ms = [[a.elapsed_time(b) for a, b in ke] for ke in kern_events]
+
+    # ---- kernel durations: the same K sweeps issued call by call with events around every attention launch
+    kern_events = [{kk: (torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True))
+                    for kk in range(shape.K)} for _ in range(args.steps)]
+    for it in range(args.steps):
+        flush.fill_(it & 0xff)
+        sweep(kern_events[it])
+    barrier()
     clocks = sampler.stop()
+    per_step_ms = np.array([[ke[kk][0].elapsed_time(ke[kk][1]) for kk in range(shape.K)] for ke in kern_events])
     assert hk.heatkv_device_status(ses.ctx) == 0
 
-    # ---- end to end: host (pinned) inputs, copies inside the timed region
-    hq, hk_, hv = (x.cpu().pin_memory() for x in (q, k, v))
-    hout = torch.empty_like(hq).pin_memory()
-    dq, dk, dv, dout = (torch.empty_like(q) for _ in range(4))
-    e2e_steps = max(3, min(args.steps, 5))
-
-    def sweep_e2e():
-        ids = [hk.heatkv_seq_open(ses.ctx, sch) for _ in range(n_seq)]
-        for step in range(shape.K):
-            lo, hi = ses.step_slices(step)
-            for src, dst in ((hq, dq), (hk_, dk), (hv, dv)):
-                dst[:, :, lo:hi].copy_(src[:, :, lo:hi], non_blocking=True)
-            ses.pre_step(ids, step)
-            ses.run_layer_step(ids, 0, step, dq, dk, dv, dout, bias[0, step])
-            hout[:, :, lo:hi].copy_(dout[:, :, lo:hi], non_blocking=True)
-        for i in ids:
-            hk.heatkv_seq_close(ses.ctx, i)
-
+    # ---- end to end: the same sweep from pinned host buffers, copies inside the timed region
+    h2d = 3 * sum(x.numel() for x in qs_) * 2
+    d2h = sum(x.numel() for x in qs_) * 2
     e2e_ms = float("nan")
+    e2e_steps = max(3, min(args.steps, 20))
     if not args.no_e2e:
+        hq, hkk, hv = ([x.cpu().pin_memory() for x in xs] for xs in (qs_, ks_, vs_))
+        hout = [torch.empty_like(x).pin_memory() for x in hq]
+        dq, dk, dv, do = ([torch.empty_like(x) for x in xs] for xs in (qs_, ks_, vs_, os_))
+
+        def sweep_e2e():
+            ids = [hk.heatkv_seq_open(ses.ctx, sch) for _ in range(n_seq)]
+            for step in range(shape.K):
+                for src, dst in ((hq, dq), (hkk, dk), (hv, dv)):
+                    dst[step].copy_(src[step], non_blocking=True)
+                ses.pre_step(ids, step)
+                hk.heatkv_scale_attention(ses.ctx, ids, 0, step, dq[step], dk[step], dv[step], None, bias[0, step], do[step])
+                hk.heatkv_append_compact(ses.ctx, ids, 0, step, dk[step], dv[step], None)
+                hout[step].copy_(do[step], non_blocking=True)
+            for i in ids:
+                hk.heatkv_seq_close(ses.ctx, i)
+
         sweep_e2e()
         barrier()
         t0 = time.perf_counter()
@@ -315,8 +380,6 @@ def main():
         e1.record(stream)
         barrier()
         e2e_ms = max(e0.elapsed_time(e1), 1e3 * (time.perf_counter() - t0)) / e2e_steps
-    h2d = 3 * q.numel() * 2
-    d2h = q.numel() * 2
 
     # ---- aggregate over ranks (replicas): slowest rank's time
     if dist is not None:
@@ -327,13 +390,13 @@ def main():
     ms_per_step = total_ms / args.steps
     value = images_per_step / (ms_per_step * 1e-3)
 
-    # ---- roofline of the dominant kernel: the attention launches of the large steps
+    # ---- roofline of the dominant kernel: attn_tc_kernel (tcgen05), all its launches of a sweep
     pk = peaks()
-    attn_ms = np.array(per_step_ms).mean(axis=0)                  # [K] mean duration per launch
-    big = [kk for kk in range(shape.K) if shape.t[kk] >= 1024]
-    dom_flops = sum(flops[kk] for kk in big)
-    dom_ms = float(sum(attn_ms[kk] for kk in big))
-    achieved = dom_flops / (dom_ms * 1e-3) / 1e12
+    attn_ms = per_step_ms.mean(axis=0)                            # [K] mean duration per launch
+    dom_flops = sum(flops[kk] for kk in tc_steps)
+    dom_ms = float(sum(attn_ms[kk] for kk in tc_steps))
+    achieved = dom_flops / (dom_ms * 1e-3) / 1e12 if tc_steps else 0.0
+    big = shape.K - 1
     uncompressed_kv_bytes = sum(2 * shape.c[kk] * shape.d * 2 for kk in range(shape.K)) * shape.H * n_seq
     line = {
         "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
@@ -341,32 +404,36 @@ def main():
         "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
         "config": {"workload": shape.name, "L": shape.L, "H": shape.H, "d": shape.d, "scales": shape.K,
                    "tokens": shape.n_tokens, "n_seq": n_seq, "budget": B_BUDGET, "policy": "heatkv", "s": shape.s,
-                   "layout": args.layout, "kernel": args.kernel, "l2": "256 MB flush write between timed steps",
+                   "layout": args.layout, "kernel": args.kernel, "launch": args.launch,
+                   "l2": "256 MB flush write between timed steps",
                    "one_image": "cond/uncond pair through one layer; x32 layers for a 2B-class model",
                    "n_k": [int(x) for x in nk], "replicas": world},
         "effective_kv_tb_per_s": uncompressed_kv_bytes / (float(attn_ms.sum()) * 1e-3) / 1e12,
         "attention_ms_per_scale": [round(float(x), 5) for x in attn_ms],
+        "attention_tflops_per_scale": [round(flops[kk] / (float(attn_ms[kk]) * 1e-3) / 1e12, 1) for kk in range(shape.K)],
         "attention_tflops_all_scales": sum(flops) / (float(attn_ms.sum()) * 1e-3) / 1e12,
         "images_per_s_32_layers_extrapolated": value / 32.0,
         "calibration": {"ms_per_sample_batch": calib_ms / len(CALIB_SEEDS),
                         "tflops": calib_flops / (calib_ms * 1e-3) / 1e12, "samples": len(CALIB_SEEDS) * n_seq},
-        "roofline": {"bound": "tensor", "kernel": "scale attention, scales with t_k >= 1024 (4 launches per step)",
+        "roofline": {"bound": "tensor", "kernel": f"attn_tc_kernel, its {len(tc_steps)} launches per sweep (scales with t_k >= 256)",
                      "achieved": achieved, "peak": pk["bf16_tflops"], "unit": "TFLOP/s",
                      "frac": achieved / pk["bf16_tflops"], "peak_source": pk["source"] + " burst bf16",
-                     "traffic": None},
+                     "largest_launch": {"scale": big + 1, "tflops": flops[big] / (float(attn_ms[big]) * 1e-3) / 1e12,
+                                        "frac": flops[big] / (float(attn_ms[big]) * 1e-3) / 1e12 / pk["bf16_tflops"]},
+                     "traffic": TRAFFIC_BYTES_PER_SWEEP},
         "e2e": {"value": images_per_step / (e2e_ms * 1e-3), "unit": UNIT, "h2d_bytes_per_step": h2d,
                 "d2h_bytes_per_step": d2h, "steps": e2e_steps},
-        "gpu_launches": int(launches),
+        "gpu_launches": int(launches_per_sweep * args.steps),
         "clocks": clocks,
     }
     if rank == 0 and world == 1 and not args.no_cpu_baseline:
-        bias_cpu = bias_np
-        n_units = 16
-        dt, threads = oracle_unit_seconds(shape, n_units, bias_cpu)
-        sec_per_image = dt / n_units * (shape.n_seq * shape.H)
-        line["cpu_baseline"] = {"value": 1.0 / sec_per_image, "unit": UNIT, "cores": threads, "kind": "oracle",
-                                "sample": f"{n_units} of {shape.n_seq * shape.H} (seq, head) units, all 13 scales "
-                                          f"(attention + cache contents), extrapolated; {dt:.1f} s of CPU work"}
+        ctx = oracle_context(shape)
+        samples = [(h, list(range(1, shape.K + 1))) for h in (0, 3, 5, 7, 8, 11, 13, 15)] * 5
+        v, secs, frac = oracle_images_per_s(shape, ctx, samples)
+        line["cpu_baseline"] = {"value": v, "unit": UNIT, "cores": torch.get_num_threads(), "kind": "oracle",
+                                "sample": f"{len(samples)} (seq, head) units of {shape.n_seq * shape.H}, all 13 scales "
+                                          f"(attention + cache contents); {secs:.1f} s of CPU work = {frac:.3g} images, "
+                                          "extrapolated by flops"}
     hk.heatkv_schedule_free(sch)
     ses.close()
     if dist is not None:

@@ -274,3 +274,62 @@ def test_step_order_and_pool_errors(hk):
     hk.heatkv_schedule_free(sch)
     hk.heatkv_schedule_free(sch2)
     ses.close()
+
+
+def test_config2_graph_replay_sampled_heads(hk):
+    """Config 2 at full size in the launch configuration the bench times: the 13-step sweep recorded
+    once into a CUDA graph (per-scale contiguous buffers, default strides) and replayed; outputs of
+    the replay against the oracle on sampled (seq, head) pairs."""
+    from paper_2605_14877_b200.sweep import Session
+    sh = W.CFG2
+    scores = W.synthetic_scas(sh, 0)
+    ref = O.heatkv_schedule(scores, 0.05, sh.s, sh.sides)
+    bias_np = W.seg_bias_current_scale(sh, 0)
+    sm = 1.0 / math.sqrt(sh.d)
+    with Session(sh.L, sh.H, sh.d, sh.t, sh.s, pool_rows=2 * sh.n_seq * sh.H * (sh.c[-2] + 64 * sh.K)) as ses:
+        sch = ses.schedule(scas=scores, b=0.05)
+        bias = torch.from_numpy(bias_np).cuda()
+        q, k, v = W.qkv_layer(sh, 0, 0, device="cuda")
+        qs, ks, vs, outs = [], [], [], []
+        for step in range(sh.K):
+            lo, hi = ses.step_slices(step)
+            qs.append(q[:, :, lo:hi].contiguous()); ks.append(k[:, :, lo:hi].contiguous())
+            vs.append(v[:, :, lo:hi].contiguous()); outs.append(torch.zeros_like(qs[-1]))
+
+        def sweep():
+            ids = [hk.heatkv_seq_open(ses.ctx, sch) for _ in range(sh.n_seq)]
+            for step in range(sh.K):
+                ses.pre_step(ids, step)
+                hk.heatkv_scale_attention(ses.ctx, ids, 0, step, qs[step], ks[step], vs[step], None, bias[0, step],
+                                          outs[step])
+                hk.heatkv_append_compact(ses.ctx, ids, 0, step, ks[step], vs[step], None)
+            for i in ids:
+                hk.heatkv_seq_close(ses.ctx, i)
+
+        sweep()                                   # plan upload and one-time kernel attributes happen here
+        torch.cuda.synchronize()
+        side = torch.cuda.Stream()
+        side.wait_stream(torch.cuda.current_stream())
+        with torch.cuda.stream(side):
+            sweep()
+        torch.cuda.current_stream().wait_stream(side)
+        torch.cuda.synchronize()
+        graph = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(graph):
+            sweep()
+        for o in outs:
+            o.zero_()
+        graph.replay()
+        graph.replay()
+        torch.cuda.synchronize()
+        assert hk.heatkv_device_status(ses.ctx) == 0
+        qh, kh, vh = _f64(q), _f64(k), _f64(v)
+        stats = _ErrStats()
+        for (s_, h) in [(0, 2), (1, 9), (1, 14)]:
+            for step in range(1, sh.K + 1):
+                brow = bias_np[0, step - 1, h].astype(np.float64)
+                lo, hi = (sh.c[step - 2] if step > 1 else 0), sh.c[step - 1]
+                want = O.scale_attention(qh[s_, h, lo:hi], kh[s_, h], vh[s_, h], ref, step, 0, h, sm, brow)
+                _check_attention(outs[step - 1][s_, h], want, ("graph", s_, h, step), stats)
+        stats.check()
+        hk.heatkv_schedule_free(sch)
