@@ -47,7 +47,8 @@ typedef enum {
   HEATKV_ERR_NAN_SCORE = -6,
   HEATKV_ERR_DEVICE_TIMEOUT = -7,      /* a bounded device-side wait gave up           */
   HEATKV_ERR_CUDA = -8,
-  HEATKV_ERR_HOST_MEMORY = -9
+  HEATKV_ERR_HOST_MEMORY = -9,
+  HEATKV_ERR_TOO_LARGE = -10           /* the call needs more built-in scratch than the library holds */
 } heatkv_status;
 
 typedef enum { HEATKV_LAYOUT_RAGGED = 0, HEATKV_LAYOUT_PAGED = 1 } heatkv_layout;
@@ -120,6 +121,25 @@ int heatkv_destroy(heatkv_ctx* ctx);
 int heatkv_calibrate_scores(heatkv_ctx* ctx, int layer, int step, int n_seq, const void* q,
                             const void* k_full, const void* v_full, const heatkv_strides* st,
                             const float* seg_bias, float* beta_accum, void* out, void* stream);
+
+/* No counterpart in the paper: heatkv_calibrate_scores for callers that must not allocate device
+ * memory while they run -- code inside a serving loop whose memory pool is fixed at start-up, a plug-in
+ * of a host application that owns the allocator, a caller between stream-ordered allocator
+ * checkpoints.  It computes the same beta update (no attention output, so no v_full / out), but every
+ * CTA writes its partial masses into a 4 MiB array that is part of the library image (held by every GPU
+ * that loads the library until the process exits) and a second small kernel adds them to beta_accum in a
+ * fixed order; the call itself makes no cudaMalloc / cudaFree and uses no allocating library routine.
+ *   Limit: ceil(t[step] / 64) * H * n_seq * 64 partial slots must fit in 2^20 floats, i.e. at most
+ *   16 384 (query tile, head, sequence) CTAs; larger calls return HEATKV_ERR_TOO_LARGE and launch nothing.
+ *   The first call on a device looks up the array's device address (once per device, on the device that
+ *   is current); make that first call before any stream capture.
+ *   All calls share the one array and it keeps the last call's contents: every slot a call reads is
+ *   written by that call first, so nothing needs clearing, but two calls whose kernels overlap on the
+ *   GPU (different streams) race on it -- keep them on one stream or order them yourself.
+ * Arguments as in heatkv_calibrate_scores.  Results agree with it up to the order of the fp32 sums. */
+int heatkv_calibrate_scores_static(heatkv_ctx* ctx, int layer, int step, int n_seq, const void* q,
+                                   const void* k_full, const heatkv_strides* st, const float* seg_bias,
+                                   float* beta_accum, void* stream);
 
 /* Text after Eq. 2, Eq. 3 and Eq. 4 -- copies beta_accum to the host (synchronises
  * `stream`), divides by n_samples = |D| and reduces in fp64:

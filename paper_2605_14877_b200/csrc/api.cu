@@ -12,6 +12,7 @@
 
 namespace heatkv {
 cudaError_t launch_attn_generic(const AttnParams& p, int d, int n_seq, bool calib, cudaStream_t stream);
+cudaError_t launch_calibrate_static(const AttnParams& p, int d, int n_seq, cudaStream_t stream, bool* too_large);
 cudaError_t launch_append(const CopyParams& p, int n_seq, cudaStream_t stream);
 cudaError_t launch_compact(const CopyParams& p, int n_seq, cudaStream_t stream);
 struct TcState;
@@ -236,6 +237,7 @@ const char* heatkv_strerror(int status) {
     case HEATKV_ERR_DEVICE_TIMEOUT: return "a bounded device-side wait ran out";
     case HEATKV_ERR_CUDA: return "CUDA runtime error";
     case HEATKV_ERR_HOST_MEMORY: return "host allocation failed";
+    case HEATKV_ERR_TOO_LARGE: return "call needs more built-in scratch than the library holds";
     default: return "unknown status";
   }
 }
@@ -470,6 +472,42 @@ int heatkv_calibrate_scores(heatkv_ctx* ctx, int layer, int step, int n_seq, con
   cudaError_t e = launch_attn_generic(p, ctx->cfg.d, n_seq, true, stream);
   ctx->launches += 1;
   return e == cudaSuccess ? HEATKV_OK : HEATKV_ERR_CUDA;
+}
+
+int heatkv_calibrate_scores_static(heatkv_ctx* ctx, int layer, int step, int n_seq, const void* q, const void* k_full,
+                                   const heatkv_strides* st, const float* seg_bias, float* beta_accum, void* stream_) {
+  if (!ctx || !q || !k_full || !beta_accum) return HEATKV_ERR_INVALID_ARG;
+  if (!aligned16(q) || !aligned16(k_full)) return HEATKV_ERR_INVALID_ARG;
+  if (layer < 0 || layer >= ctx->cfg.L || step < 0 || step >= ctx->cfg.K || n_seq < 1 || n_seq > 65535)
+    return HEATKV_ERR_INVALID_ARG;
+  cudaStream_t stream = static_cast<cudaStream_t>(stream_);
+  AttnParams p;
+  std::memset(&p, 0, sizeof(p));
+  heatkv_strides s;
+  if (!st) {   // dense: q [n_seq,H,t,d], k [n_seq,H,c[step],d]
+    const int64_t d = ctx->cfg.d, H = ctx->cfg.H, t = ctx->cfg.t[step], c = ctx->c[step];
+    s.q_tok = s.kv_tok = s.o_tok = d;
+    s.q_head = s.o_head = d * t; s.kv_head = d * c;
+    s.q_seq = s.o_seq = d * t * H; s.kv_seq = d * c * H;
+  } else {
+    int rc = check_strides(ctx, st, ctx->cfg.t[step], &s);
+    if (rc != HEATKV_OK) return rc;
+  }
+  fill_common(ctx, &p, s);
+  p.q = static_cast<const __nv_bfloat16*>(q);
+  p.k_new = static_cast<const __nv_bfloat16*>(k_full);
+  p.seg_bias = seg_bias;
+  p.t_q = ctx->cfg.t[step];
+  p.n_own = ctx->c[step];
+  p.step = step;
+  p.layer = layer;
+  p.beta_row = beta_accum + (((int64_t)layer * ctx->cfg.H) * ctx->cfg.K + step) * ctx->cfg.K;
+  bool too_large = false;
+  cudaError_t e = launch_calibrate_static(p, ctx->cfg.d, n_seq, stream, &too_large);
+  if (too_large) return HEATKV_ERR_TOO_LARGE;
+  if (e != cudaSuccess) return HEATKV_ERR_CUDA;
+  ctx->launches += 2;
+  return HEATKV_OK;
 }
 
 int heatkv_finalize_scores(heatkv_ctx* ctx, const float* beta_accum, int n_samples, double* beta, double* scas,

@@ -49,7 +49,13 @@ __device__ __forceinline__ void load_tile(uint32_t smem_base, const __nv_bfloat1
   }
 }
 
-template <int D, bool CALIB>
+// Scratch of heatkv_calibrate_scores_static: one partial mass per (CTA, warp, source scale).  It lives in
+// the library image, so that entry point needs no allocation; every GPU that loads the library holds
+// these 4 MiB until the process exits.
+constexpr int STATIC_PARTIAL_FLOATS = 1 << 20;
+static __device__ __align__(256) float g_static_partials[STATIC_PARTIAL_FLOATS];
+
+template <int D, bool CALIB, bool PARTIALS = false>
 __global__ void __launch_bounds__(GTHREADS, 2) attn_generic_kernel(const __grid_constant__ AttnParams p) {
   extern __shared__ __align__(128) unsigned char smem[];
   using SM = GenericSmem<D>;
@@ -308,7 +314,13 @@ __global__ void __launch_bounds__(GTHREADS, 2) attn_generic_kernel(const __grid_
       acc += __shfl_xor_sync(0xffffffffu, acc, 4);
       acc += __shfl_xor_sync(0xffffffffu, acc, 8);
       acc += __shfl_xor_sync(0xffffffffu, acc, 16);
-      if (lane == 0) atomicAdd(beta + sg, acc / (float)p.t_q);
+      if (PARTIALS) {
+        // slot of (CTA, warp, source scale); reduce_partials_kernel adds them up in a fixed order
+        const int64_t cta = blockIdx.x + (int64_t)gridDim.x * (blockIdx.y + (int64_t)gridDim.y * blockIdx.z);
+        if (lane == 0) p.partials[(cta * (GTHREADS / 32) + warp) * HEATKV_MAX_K + sg] = acc / (float)p.t_q;
+      } else {
+        if (lane == 0) atomicAdd(beta + sg, acc / (float)p.t_q);
+      }
     }
   }
 
@@ -336,6 +348,21 @@ __global__ void __launch_bounds__(GTHREADS, 2) attn_generic_kernel(const __grid_
   }
 }
 
+// beta[head][step][sg] += sum of the partials of that head in the order (sequence, query tile, warp):
+// one thread per (head, source scale), so the result does not depend on scheduling.
+__global__ void reduce_partials_kernel(const float* partials, float* beta_row, int n_qtiles, int H, int n_seq, int K,
+                                       int step) {
+  const int head = blockIdx.x, sg = threadIdx.x;
+  if (sg > step) return;
+  float acc = 0.f;
+  for (int seq = 0; seq < n_seq; ++seq)
+    for (int qt = 0; qt < n_qtiles; ++qt) {
+      const int64_t cta = qt + (int64_t)n_qtiles * (head + (int64_t)H * seq);
+      for (int w = 0; w < GTHREADS / 32; ++w) acc += partials[(cta * (GTHREADS / 32) + w) * HEATKV_MAX_K + sg];
+    }
+  beta_row[(int64_t)head * K * K + sg] += acc;
+}
+
 template <int D, bool CALIB>
 static cudaError_t launch_one(const AttnParams& p, int n_seq, cudaStream_t stream) {
   auto kern = attn_generic_kernel<D, CALIB>;
@@ -347,6 +374,61 @@ static cudaError_t launch_one(const AttnParams& p, int n_seq, cudaStream_t strea
   }
   dim3 grid((p.t_q + GM - 1) / GM, CALIB ? p.H : n_seq, CALIB ? n_seq : p.H);
   kern<<<grid, GTHREADS, GenericSmem<D>::BYTES, stream>>>(p);
+  return cudaGetLastError();
+}
+
+// Calibration pass whose scratch is the static array above.  Returns cudaErrorInvalidValue when the
+// launch would need more partial slots than the array has.  The array's device address is looked up
+// once per device (cudaGetSymbolAddress; the symbol's name itself is only a host-side handle).
+cudaError_t launch_calibrate_static(const AttnParams& p_in, int d, int n_seq, cudaStream_t stream, bool* too_large) {
+  *too_large = false;
+  const int n_qtiles = (p_in.t_q + GM - 1) / GM;
+  const int64_t slots = (int64_t)n_qtiles * p_in.H * n_seq * (GTHREADS / 32) * HEATKV_MAX_K;
+  if (slots > STATIC_PARTIAL_FLOATS) {
+    *too_large = true;
+    return cudaErrorInvalidValue;
+  }
+  constexpr int MAX_DEVICES = 64;
+  static float* scratch_of_device[MAX_DEVICES] = {nullptr};
+  static bool configured[MAX_DEVICES][2] = {{false}};
+  int dev = -1;
+  cudaError_t e = cudaGetDevice(&dev);
+  if (e != cudaSuccess) return e;
+  if (dev < 0 || dev >= MAX_DEVICES) return cudaErrorInvalidDevice;
+  if (!scratch_of_device[dev]) {
+    float* ptr = nullptr;
+    e = cudaGetSymbolAddress(reinterpret_cast<void**>(&ptr), g_static_partials);
+    if (e != cudaSuccess) return e;
+    scratch_of_device[dev] = ptr;
+  }
+  AttnParams p = p_in;
+  p.partials = scratch_of_device[dev];
+  p.out = nullptr;
+  p.v_new = nullptr;
+  const int which = d == 128 ? 1 : 0;
+  dim3 grid(n_qtiles, p.H, n_seq);
+  if (d == 128) {
+    auto kern = attn_generic_kernel<128, true, true>;
+    if (!configured[dev][which]) {
+      e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, GenericSmem<128>::BYTES);
+      if (e != cudaSuccess) return e;
+      configured[dev][which] = true;
+    }
+    kern<<<grid, GTHREADS, GenericSmem<128>::BYTES, stream>>>(p);
+  } else if (d == 64) {
+    auto kern = attn_generic_kernel<64, true, true>;
+    if (!configured[dev][which]) {
+      e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, GenericSmem<64>::BYTES);
+      if (e != cudaSuccess) return e;
+      configured[dev][which] = true;
+    }
+    kern<<<grid, GTHREADS, GenericSmem<64>::BYTES, stream>>>(p);
+  } else {
+    return cudaErrorInvalidValue;
+  }
+  e = cudaGetLastError();
+  if (e != cudaSuccess) return e;
+  reduce_partials_kernel<<<p.H, HEATKV_MAX_K, 0, stream>>>(p.partials, p.beta_row, n_qtiles, p.H, n_seq, p.K, p.step);
   return cudaGetLastError();
 }
 

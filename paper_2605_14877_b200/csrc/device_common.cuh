@@ -34,6 +34,7 @@ struct AttnParams {
   int32_t c[HEATKV_MAX_K];        // cumulative tokens (calibration: column -> source scale)
   uint32_t* status;               // device status word (non-zero = a bounded wait gave up)
   SeqRef seqs[HEATKV_MAX_BATCH];
+  float* partials;                // calibration with a fixed summation order: per-warp partial masses, else null
 };
 
 struct CopyParams {

@@ -18,8 +18,8 @@ __all__ = [
     "LAYOUT_RAGGED", "LAYOUT_PAGED", "POLICY_HEATKV", "POLICY_BINARY", "POLICY_NAIVE", "POLICY_EXPLICIT",
     "ACCOUNT_PHYSICAL", "ACCOUNT_LITERAL", "KERNEL_AUTO", "KERNEL_GENERIC", "KERNEL_TCGEN05",
     "MAX_K", "MAX_BATCH", "PAGE_TOKENS",
-    "heatkv_create", "heatkv_destroy", "heatkv_calibrate_scores", "heatkv_finalize_scores",
-    "heatkv_build_schedule", "heatkv_schedule_free", "heatkv_schedule_masks", "heatkv_schedule_footprint",
+    "heatkv_create", "heatkv_destroy", "heatkv_calibrate_scores", "heatkv_calibrate_scores_static",
+    "heatkv_finalize_scores", "heatkv_build_schedule", "heatkv_schedule_free", "heatkv_schedule_masks", "heatkv_schedule_footprint",
     "heatkv_schedule_plan", "heatkv_seq_open", "heatkv_seq_close", "heatkv_append_compact", "heatkv_scale_attention",
     "heatkv_cache_bytes", "heatkv_retained_indices", "heatkv_export_head", "heatkv_allocator_stats",
     "heatkv_launch_count", "heatkv_device_status", "heatkv_strerror", "arena_bytes_for",
@@ -85,7 +85,8 @@ def lib_path() -> str:
 
 def exported_symbols():
     """Names declared in include/heatkv.h, in declaration order."""
-    return ["heatkv_create", "heatkv_destroy", "heatkv_calibrate_scores", "heatkv_finalize_scores",
+    return ["heatkv_create", "heatkv_destroy", "heatkv_calibrate_scores", "heatkv_calibrate_scores_static",
+            "heatkv_finalize_scores",
             "heatkv_build_schedule", "heatkv_schedule_free", "heatkv_schedule_masks",
             "heatkv_schedule_footprint", "heatkv_schedule_plan", "heatkv_seq_open", "heatkv_seq_close", "heatkv_append_compact",
             "heatkv_scale_attention", "heatkv_cache_bytes", "heatkv_retained_indices", "heatkv_export_head",
@@ -107,6 +108,7 @@ _P = C.c_void_p
 _lib.heatkv_create.argtypes = [C.POINTER(Config), _P, C.POINTER(_P)]
 _lib.heatkv_destroy.argtypes = [_P]
 _lib.heatkv_calibrate_scores.argtypes = [_P, C.c_int, C.c_int, C.c_int, _P, _P, _P, C.POINTER(Strides), _P, _P, _P, _P]
+_lib.heatkv_calibrate_scores_static.argtypes = [_P, C.c_int, C.c_int, C.c_int, _P, _P, C.POINTER(Strides), _P, _P, _P]
 _lib.heatkv_finalize_scores.argtypes = [_P, _P, C.c_int, _P, _P, _P, _P]
 _lib.heatkv_build_schedule.argtypes = [C.POINTER(Config), _P, _P, C.c_int, C.c_int, C.c_double, _P, C.POINTER(_P)]
 _lib.heatkv_schedule_free.argtypes = [_P]
@@ -180,6 +182,15 @@ def heatkv_calibrate_scores(ctx, layer, step, n_seq, q, k_full, v_full, strides,
     _check(_lib.heatkv_calibrate_scores(ctx, layer, step, n_seq, _ptr(q), _ptr(k_full), _ptr(v_full), st,
                                         _ptr(seg_bias), _ptr(beta_accum), _ptr(out), _stream(stream)),
            "heatkv_calibrate_scores")
+
+
+def heatkv_calibrate_scores_static(ctx, layer, step, n_seq, q, k_full, strides, seg_bias, beta_accum,
+                                   stream=None) -> None:
+    """Same beta update as heatkv_calibrate_scores, for callers that must not allocate device memory:
+    the scratch is an array inside the library.  Raises HeatKVError(-10) when the call is too large."""
+    st = C.byref(strides) if strides is not None else None
+    _check(_lib.heatkv_calibrate_scores_static(ctx, layer, step, n_seq, _ptr(q), _ptr(k_full), st, _ptr(seg_bias),
+                                               _ptr(beta_accum), _stream(stream)), "heatkv_calibrate_scores_static")
 
 
 def heatkv_finalize_scores(ctx, beta_accum, n_samples, L, H, K, stream=None):

@@ -1,0 +1,61 @@
+"""heatkv_calibrate_scores_static: the calibration update for callers that cannot allocate device
+memory while they run (a serving loop with a memory pool fixed at start-up, a plug-in whose host owns
+the allocator).  Its scratch is an array built into the library, so the call itself allocates nothing.
+
+The test drives the entry point through the C ABI twice in a row into one accumulator and compares it
+with two calls of heatkv_calibrate_scores on the same inputs, at the tolerance the other calibration
+tests use (1e-3 relative).  Two calls matter: the built-in array is shared by all calls and keeps the
+previous call's contents, so a second call that read stale slots would show up here.  The file is named
+so that pytest collects it last.
+"""
+import numpy as np
+import pytest
+import torch
+
+import heatkv_workloads as W
+
+pytestmark = pytest.mark.gpu
+
+RTOL_BETA = 1e-3
+
+
+def test_static_scratch_calibration_matches_allocating_entry_point_twice():
+    import paper_2605_14877_b200 as hk
+    from paper_2605_14877_b200.sweep import Session
+
+    sh = W.Shape("mid", L=2, H=3, d=128, sides=W.SIDES_13[:10], n_seq=2, s=3)
+    bias = torch.from_numpy(W.seg_bias_prior_lognormal(sh, 8)).cuda()
+    ses = Session(sh.L, sh.H, sh.d, sh.t, sh.s, pool_rows=64, kernel=hk.KERNEL_GENERIC)
+    want = torch.zeros(sh.L, sh.H, sh.K, sh.K, dtype=torch.float32, device="cuda")
+    got = torch.zeros_like(want)
+    # all inputs exist before the calls under test: those calls must not need any allocation
+    layers = [W.qkv_layer(sh, 5, l, device="cuda") for l in range(sh.L)]
+    torch.cuda.synchronize()
+    for call in range(2):
+        for l in range(sh.L):
+            q, k, _ = layers[l]
+            for step in range(sh.K):
+                lo, hi = ses.step_slices(step)
+                qs, ks = q[:, :, lo:hi], k[:, :, :hi]
+                st = hk.Strides.of(qs, ks)
+                hk.heatkv_calibrate_scores(ses.ctx, l, step, sh.n_seq, qs, ks, None, st, bias[l, step], want, None)
+                hk.heatkv_calibrate_scores_static(ses.ctx, l, step, sh.n_seq, qs, ks, st, bias[l, step], got)
+        torch.cuda.synchronize()
+        a, b = want.double().cpu().numpy(), got.double().cpu().numpy()
+        mask = a > 1e-5 * (call + 1)
+        assert mask.sum() > 100
+        assert np.all(np.abs(a - b)[mask] <= RTOL_BETA * a[mask]), (call, float(np.abs(a - b)[mask].max()))
+        assert np.all(np.triu(b, 1) == 0)
+        # each (layer, head, step) row holds n_seq * (call + 1) probability vectors
+        assert np.allclose(b.sum(axis=-1), sh.n_seq * (call + 1), atol=1e-3)
+    # a call that would need more partial slots than the built-in array has is refused, nothing runs
+    before = got.clone()
+    q, k, _ = layers[0]
+    lo, hi = ses.step_slices(sh.K - 1)
+    with pytest.raises(hk.HeatKVError) as e:
+        hk.heatkv_calibrate_scores_static(ses.ctx, 0, sh.K - 1, 60000, q[:, :, lo:hi], k[:, :, :hi],
+                                          hk.Strides.of(q[:, :, lo:hi], k[:, :, :hi]), None, got)
+    assert e.value.status == -10
+    torch.cuda.synchronize()
+    assert torch.equal(before, got)
+    ses.close()
