@@ -21,6 +21,12 @@ void tc_destroy(TcState* st);
 bool tc_supported(const TcState* st, const AttnParams& p, int d, int n_seq, bool calib);
 cudaError_t launch_attn_tc(TcState* st, const AttnParams& p, int d, int n_seq, bool calib, cudaStream_t stream,
                            int* launches);
+struct CalibTcState;
+uint64_t calib_tc_desc_bytes(const heatkv_config& cfg);
+int calib_tc_create(const heatkv_config& cfg, void* dev_table, cudaStream_t stream, CalibTcState** out);
+void calib_tc_destroy(CalibTcState* st);
+bool calib_tc_supported(const CalibTcState* st, const AttnParams& p, int d, int n_seq);
+cudaError_t launch_calib_tc(CalibTcState* st, const AttnParams& p, int n_seq, cudaStream_t stream);
 }  // namespace heatkv
 
 using namespace heatkv;
@@ -105,6 +111,7 @@ struct heatkv_ctx {
   uint64_t reserved_rows = 0, peak_reserved = 0, meta_used = 0;
   uint64_t launches = 0;
   TcState* tc = nullptr;
+  CalibTcState* calib_tc = nullptr;
 };
 
 namespace {
@@ -281,6 +288,21 @@ int heatkv_create(const heatkv_config* cfg, void* stream_, heatkv_ctx** out) {
   if (cudaMemsetAsync(ctx->k_pool, 0, 2 * rows * row_bytes, stream) != cudaSuccess) return HEATKV_ERR_CUDA;
   int rc = tc_create(ctx->cfg, ctx->k_pool, ctx->v_pool, rows, &ctx->tc);
   if (rc != HEATKV_OK) return rc;
+  // the calibration kernel's half-tile table (key rows cut at source-scale borders) sits in the metadata region
+  void* calib_table = nullptr;
+  {
+    uint64_t bytes = (calib_tc_desc_bytes(ctx->cfg) + META_ALIGN - 1) / META_ALIGN * META_ALIGN, off = 0;
+    if (bytes && ctx->metas.alloc(bytes, &off)) {
+      calib_table = ctx->meta + off;
+      ctx->meta_used += bytes;
+    }
+  }
+  rc = calib_tc_create(ctx->cfg, calib_table, stream, &ctx->calib_tc);
+  if (rc != HEATKV_OK) {
+    tc_destroy(ctx->tc);
+    calib_tc_destroy(ctx->calib_tc);
+    return rc;
+  }
   *out = ctx.release();
   return HEATKV_OK;
 }
@@ -288,6 +310,7 @@ int heatkv_create(const heatkv_config* cfg, void* stream_, heatkv_ctx** out) {
 int heatkv_destroy(heatkv_ctx* ctx) {
   if (!ctx) return HEATKV_ERR_INVALID_ARG;
   tc_destroy(ctx->tc);
+  calib_tc_destroy(ctx->calib_tc);
   delete ctx;
   return HEATKV_OK;
 }
@@ -469,7 +492,12 @@ int heatkv_calibrate_scores(heatkv_ctx* ctx, int layer, int step, int n_seq, con
   p.step = step;
   p.layer = layer;
   p.beta_row = beta_accum + (((int64_t)layer * ctx->cfg.H) * ctx->cfg.K + step) * ctx->cfg.K;
-  cudaError_t e = launch_attn_generic(p, ctx->cfg.d, n_seq, true, stream);
+  // without an attention output the pass is S = Q K^T plus bookkeeping: the tensor-memory kernel takes it
+  const int choice = ctx->cfg.kernel;
+  bool use_tc = !out && choice != HEATKV_KERNEL_GENERIC && calib_tc_supported(ctx->calib_tc, p, ctx->cfg.d, n_seq);
+  if (choice == HEATKV_KERNEL_AUTO && p.t_q < 256) use_tc = false;
+  cudaError_t e = use_tc ? launch_calib_tc(ctx->calib_tc, p, n_seq, stream)
+                         : launch_attn_generic(p, ctx->cfg.d, n_seq, true, stream);
   ctx->launches += 1;
   return e == cudaSuccess ? HEATKV_OK : HEATKV_ERR_CUDA;
 }

@@ -1,0 +1,438 @@
+// Tensor-memory calibration kernel (Sec. 3.1, Eq. 2) for the large scale steps (head_dim 128).
+//
+// beta[step][i] needs, for every query row of the step, the share of its softmax mass that falls on
+// the keys of source scale i.  Only S = Q K^T is a contraction here: there is no PV product and no
+// output, so the kernel is the attention kernel's front half with the per-scale bookkeeping fused into
+// the softmax pass; the attention matrix is never written anywhere.
+//
+// One CTA owns 256 queries of one (sequence, head) as two 128-row tiles A and B.  Warp roles:
+//   warp 0      TMA producer: Q tiles once, then K half-tiles (64 rows x 128 dims) of the full key set,
+//               cut at source-scale borders (descriptor list built on the host), 4 stages.
+//   warp 1      MMA issuer: S_x = Q_x K^T into TMEM as soon as the softmax warps have read the
+//               previous S_x into registers (they say so right after the load, before the exponentials).
+//   warps 4-7   tile A, warps 8-11 tile B: one thread per query row keeps the running max, the row sum
+//               and the mass of the scale it is inside; finished scales are parked in shared memory
+//               relative to the same reference and rescaled when the reference moves (rare).
+// At the end every row's masses are divided by its row sum, summed over the CTA's rows and added to
+// beta with one atomicAdd per (CTA, source scale).  Every wait is bounded as in the attention kernel.
+#include <new>
+#include <vector>
+
+#include "internal.h"
+#include "tc_common.cuh"
+
+namespace heatkv {
+
+namespace calib {
+
+using namespace tc;
+
+constexpr int D = 128;
+constexpr int BM = 128;                 // rows per Q tile
+constexpr int BN = 128;                 // keys per tile (two 64-row half-tiles)
+constexpr int HALF = 64;
+constexpr int THREADS = 384;
+constexpr int K_STAGES = 4;
+constexpr uint32_t HALF_COLS_BYTES = 128 * 128;        // one 64-column half of a 128-row tile: 16 KB
+constexpr uint32_t TILE_BYTES = 2 * HALF_COLS_BYTES;   // 32 KB
+constexpr uint32_t SLOT_BYTES = HALF * 128;            // 64 rows x 128 B inside one column half
+
+constexpr uint32_t SM_Q = 0;                                   // 2 tiles
+constexpr uint32_t SM_K = SM_Q + 2 * TILE_BYTES;               // K_STAGES tiles
+constexpr uint32_t SM_SEG = SM_K + K_STAGES * TILE_BYTES;      // float[2 tiles][16 scales][128 rows]
+constexpr uint32_t SM_ACC = SM_SEG + 2 * HEATKV_MAX_K * BM * 4;  // float[16]: the CTA's sums per scale
+constexpr uint32_t SM_BAR = SM_ACC + HEATKV_MAX_K * 4;
+constexpr uint32_t SM_TOTAL = SM_BAR + 256;
+constexpr uint32_t SM_ALLOC = SM_TOTAL + 1024;                 // slack for manual alignment
+
+enum Bar : uint32_t {
+  Q_FULL = 0,                   // +x (2)
+  K_FULL = 2, K_EMPTY = 6,      // +stage (4 each)
+  S_FULL = 10,                  // +x  S_x of tile j is in TMEM
+  S_READ = 12,                  // +x  the 128 rows of S_x of tile j are in registers (128 arrivals)
+  N_BARS = 14
+};
+constexpr uint32_t SM_TMEM_PTR = SM_BAR + N_BARS * 8;
+constexpr uint32_t SM_ABORT = SM_TMEM_PTR + 4;
+constexpr uint32_t TMEM_COLS = 256;
+
+struct Maps {
+  CUtensorMap q, k;
+};
+
+struct HalfTile {
+  int row;          // first key row inside k_full
+  int n_valid;      // real rows of the 64
+  int seg;          // source scale
+};
+
+__device__ __forceinline__ HalfTile get_half(int i, const int2* descs, int n_slots) {
+  const bool valid = i < n_slots;
+  const int2 d = descs[valid ? i : n_slots - 1];     // padding half-tile: re-read finite data, mask everything
+  HalfTile h;
+  h.row = d.x;
+  h.n_valid = valid ? (d.y & 0xff) : 0;
+  h.seg = (d.y >> 8) & 0xff;
+  return h;
+}
+
+__global__ void __launch_bounds__(THREADS, 1)
+calib_tc_kernel(const __grid_constant__ AttnParams p, const __grid_constant__ Maps maps, const int2* __restrict__ descs,
+                int n_slots) {
+  extern __shared__ unsigned char smem_raw[];
+  const uint32_t raw = smem_u32(smem_raw);
+  const uint32_t sbase = (raw + 1023u) & ~1023u;
+  unsigned char* sgen = smem_raw + (sbase - raw);
+  volatile uint32_t* abort_flag = reinterpret_cast<volatile uint32_t*>(sgen + SM_ABORT);
+  volatile uint32_t* tmem_ptr_smem = reinterpret_cast<volatile uint32_t*>(sgen + SM_TMEM_PTR);
+  float* acc_smem = reinterpret_cast<float*>(sgen + SM_ACC);
+  auto bar = [&](uint32_t which) { return sbase + SM_BAR + which * 8; };
+
+  const int warp = __shfl_sync(0xffffffffu, (int)(threadIdx.x >> 5), 0), lane = threadIdx.x & 31;
+  const int seq = blockIdx.y, head = blockIdx.z;
+  const int q0 = blockIdx.x * (2 * BM);
+  const int nq = (q0 + BM < p.t_q) ? 2 : 1;          // does tile B hold any query?
+  const int n_tiles = (n_slots + 1) / 2;
+
+  if (threadIdx.x == 0) {
+    *abort_flag = *reinterpret_cast<volatile uint32_t*>(p.status) != 0;   // an earlier CTA gave up: do not wait again
+    for (int i = 0; i < HEATKV_MAX_K; ++i) acc_smem[i] = 0.f;
+    for (int x = 0; x < 2; ++x) {
+      mbar_init(bar(Q_FULL + x), 1);
+      mbar_init(bar(S_FULL + x), 1);
+      mbar_init(bar(S_READ + x), BM);
+    }
+    for (int s = 0; s < K_STAGES; ++s) {
+      mbar_init(bar(K_FULL + s), 1);
+      mbar_init(bar(K_EMPTY + s), 1);
+    }
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+  }
+  if (warp == 0) {
+    __syncwarp();
+    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(sbase + SM_TMEM_PTR), "r"(TMEM_COLS)
+                 : "memory");
+    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+  }
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  const uint32_t tmem = *tmem_ptr_smem;
+
+  // register budget per warpgroup: 128*72 + 256*216 <= 384*168
+  if (warp < 4) {
+    reg_dealloc<72>();
+    if (warp == 0) {
+      // ------------------------------------------------------------------ TMA producer
+      const bool leader = elect_one();
+      uint32_t armed = 0;                               // stage -> a copy was issued at least once
+      uint32_t par[K_STAGES] = {0, 0, 0, 0};
+      if (leader) {
+        for (int x = 0; x < nq; ++x) {
+          mbar_expect_tx(bar(Q_FULL + x), TILE_BYTES);
+          for (int ch = 0; ch < 2; ++ch)
+            for (int hf = 0; hf < 2; ++hf)
+              tma_load_4d(sbase + SM_Q + x * TILE_BYTES + ch * HALF_COLS_BYTES + hf * SLOT_BYTES, &maps.q, ch * 64,
+                          q0 + x * BM + hf * HALF, head, seq, bar(Q_FULL + x));
+        }
+      }
+      bool ok = true;
+      for (int j = 0; j < n_tiles && ok; ++j) {
+        const int st = j % K_STAGES;
+        const uint32_t use = (uint32_t)(j / K_STAGES);
+        const HalfTile h0 = get_half(2 * j, descs, n_slots), h1 = get_half(2 * j + 1, descs, n_slots);
+        if (use > 0) ok = warp_wait(bar(K_EMPTY + st), (use - 1) & 1, abort_flag, p.status);
+        if (!ok) break;
+        armed |= 1u << st;
+        par[st] = use & 1;
+        if (leader) {
+          mbar_expect_tx(bar(K_FULL + st), TILE_BYTES);
+          for (int hf = 0; hf < 2; ++hf)
+            for (int ch = 0; ch < 2; ++ch)
+              tma_load_4d(sbase + SM_K + st * TILE_BYTES + ch * HALF_COLS_BYTES + hf * SLOT_BYTES, &maps.k, ch * 64,
+                          hf == 0 ? h0.row : h1.row, head, seq, bar(K_FULL + st));
+        }
+        __syncwarp();
+      }
+      if (!ok) {
+        // leaving early: let every copy this warp started land before the CTA exits
+        for (int s = 0; s < K_STAGES; ++s)
+          if (armed & (1u << s))
+            for (uint32_t it = 0; it < WAIT_LIMIT && !mbar_try(bar(K_FULL + s), par[s]); ++it) {}
+        for (int x = 0; x < nq; ++x)
+          for (uint32_t it = 0; it < WAIT_LIMIT && !mbar_try(bar(Q_FULL + x), 0); ++it) {}
+      }
+    } else if (warp == 1) {
+      // ------------------------------------------------------------------ MMA issuer
+      const bool leader = elect_one();
+      constexpr uint32_t IDESC_S = instr_desc(BM, BN, 0, 0);     // Q, K both K-major
+      bool ok = true;
+      for (int x = 0; x < nq && ok; ++x) ok = warp_wait(bar(Q_FULL + x), 0, abort_flag, p.status);
+      for (int j = 0; j < n_tiles && ok; ++j) {
+        const int st = j % K_STAGES;
+        ok = warp_wait(bar(K_FULL + st), (uint32_t)(j / K_STAGES) & 1, abort_flag, p.status);
+        for (int x = 0; x < nq && ok; ++x) {
+          if (j > 0) ok = warp_wait(bar(S_READ + x), (j - 1) & 1, abort_flag, p.status);
+          if (!ok) break;
+          tc_fence_after();
+          if (leader) {
+            const uint32_t qa = sbase + SM_Q + x * TILE_BYTES, ka = sbase + SM_K + st * TILE_BYTES;
+#pragma unroll
+            for (int ks = 0; ks < D / 16; ++ks) {
+              const uint32_t off = (ks >> 2) * HALF_COLS_BYTES + (ks & 3) * 32;
+              mma_ss(tmem + x * 128, smem_desc(qa + off, 16, 1024), smem_desc(ka + off, 16, 1024), IDESC_S, ks > 0);
+            }
+            tc_commit(bar(S_FULL + x));
+          }
+          __syncwarp();
+        }
+        if (ok && leader) tc_commit(bar(K_EMPTY + st));
+        __syncwarp();
+      }
+    }
+  } else {
+    reg_alloc<216>();
+    // ------------------------------------------------------------------ softmax with per-scale masses
+    const int x = (warp - 4) >> 2;                      // 0: tile A, 1: tile B
+    if (x < nq) {
+      const int row = (warp & 3) * 32 + lane;           // row inside the tile == TMEM lane
+      const uint32_t t_s = tmem + ((uint32_t)((warp & 3) * 32) << 16) + x * 128;
+      float* seg_smem = reinterpret_cast<float*>(sgen + SM_SEG) + x * (HEATKV_MAX_K * BM);   // [scale][row]
+      const float* bias_h = p.seg_bias ? p.seg_bias + head * p.K : nullptr;
+      const float LOG2E = 1.4426950408889634f;
+      float m_ref = -INFINITY, l_sum = 0.f;
+      int cur_seg = -1;                                 // the scale whose mass is being collected (warp-uniform)
+      float cur_sum = 0.f;
+      bool ok = true;
+      for (int j = 0; j < n_tiles && ok; ++j) {
+        const HalfTile s0 = get_half(2 * j, descs, n_slots), s1 = get_half(2 * j + 1, descs, n_slots);
+        const float b0 = bias_h ? bias_h[s0.seg] * LOG2E : 0.f;
+        const float b1 = bias_h ? bias_h[s1.seg] * LOG2E : 0.f;
+        ok = __all_sync(0xffffffffu, mbar_wait(bar(S_FULL + x), j & 1, abort_flag, p.status));
+        if (!ok) break;
+        tc_fence_after();
+        uint32_t r0[32], r1[32], r2[32], r3[32];
+        tmem_ld32(t_s, r0);
+        tmem_ld32(t_s + 32, r1);
+        tmem_ld32(t_s + 64, r2);
+        tmem_ld32(t_s + 96, r3);
+        tmem_wait_ld();
+        tc_fence_before();
+        mbar_arrive(bar(S_READ + x));                   // the next S_x may overwrite these columns
+        if (s0.n_valid < HALF || s1.n_valid < HALF) {   // ragged tile (warp-uniform): mask by -inf
+#pragma unroll
+          for (int i = 0; i < 32; ++i) {
+            if (i >= s0.n_valid) r0[i] = 0xff800000u;
+            if (i + 32 >= s0.n_valid) r1[i] = 0xff800000u;
+            if (i >= s1.n_valid) r2[i] = 0xff800000u;
+            if (i + 32 >= s1.n_valid) r3[i] = 0xff800000u;
+          }
+        }
+        // row maximum: the logit is raw * scale + bias(half) with scale > 0, so take the raw maxima
+        float mq[8];
+#pragma unroll
+        for (int c = 0; c < 4; ++c) {
+          mq[c] = fmaxf(__uint_as_float(r0[c]), __uint_as_float(r1[c]));
+          mq[4 + c] = fmaxf(__uint_as_float(r2[c]), __uint_as_float(r3[c]));
+        }
+#pragma unroll
+        for (int i = 4; i < 32; i += 4) {
+#pragma unroll
+          for (int c = 0; c < 4; ++c) {
+            mq[c] = fmax3(mq[c], __uint_as_float(r0[i + c]), __uint_as_float(r1[i + c]));
+            mq[4 + c] = fmax3(mq[4 + c], __uint_as_float(r2[i + c]), __uint_as_float(r3[i + c]));
+          }
+        }
+        const float mx0 = fmaxf(fmaxf(mq[0], mq[1]), fmaxf(mq[2], mq[3]));
+        const float mx1 = fmaxf(fmaxf(mq[4], mq[5]), fmaxf(mq[6], mq[7]));
+        const float mx = fmaxf(fmaf(mx0, p.scale_log2, b0), fmaf(mx1, p.scale_log2, b1));
+        const float m_new = fmaxf(m_ref, mx);
+        const bool grow = m_new > m_ref + RESCALE_THRESHOLD;   // also true on the first tile (m_ref = -inf)
+        if (grow) {
+          if (j > 0) {
+            // everything collected so far is relative to m_ref: move it to the new reference
+            const float f = exp2f(m_ref - m_new);
+            l_sum *= f;
+            cur_sum *= f;
+            for (int s = 0; s < cur_seg; ++s) seg_smem[s * BM + row] *= f;
+          }
+          m_ref = m_new;
+        }
+        __syncwarp();
+        const uint64_t scale2 = pack2(p.scale_log2, p.scale_log2);
+        auto exp_sum = [&](const uint32_t (&rc)[32], uint64_t bb2, uint64_t& sum2) {
+#pragma unroll
+          for (int i = 0; i < 32; i += 2) {
+            const uint64_t xx = fma2(pack2(__uint_as_float(rc[i]), __uint_as_float(rc[i + 1])), scale2, bb2);
+            float e0, e1;
+            if (((i >> 1) & POLY_MASK) == POLY_MASK) {
+              exp2_poly2(xx, e0, e1);
+            } else {
+              float x0, x1;
+              unpack2(xx, x0, x1);
+              e0 = ex2_approx(x0);
+              e1 = ex2_approx(x1);
+            }
+            sum2 = add2(sum2, pack2(e0, e1));
+          }
+        };
+        const uint64_t bb0 = pack2(b0 - m_ref, b0 - m_ref), bb1 = pack2(b1 - m_ref, b1 - m_ref);
+        uint64_t sum_h0 = pack2(0.f, 0.f), sum_h1 = pack2(0.f, 0.f);
+        exp_sum(r0, bb0, sum_h0);
+        exp_sum(r1, bb0, sum_h0);
+        exp_sum(r2, bb1, sum_h1);
+        exp_sum(r3, bb1, sum_h1);
+        float a0, a1, c0, c1;
+        unpack2(sum_h0, a0, a1);
+        unpack2(sum_h1, c0, c1);
+        const float h0 = a0 + a1, h1 = c0 + c1;
+        l_sum += h0 + h1;
+        // source scales arrive in ascending order, each as one run of half-tiles
+        if (s0.seg != cur_seg) {
+          if (cur_seg >= 0) seg_smem[cur_seg * BM + row] = cur_sum;
+          cur_seg = s0.seg;
+          cur_sum = 0.f;
+        }
+        cur_sum += h0;
+        if (s1.n_valid > 0) {
+          if (s1.seg != cur_seg) {
+            seg_smem[cur_seg * BM + row] = cur_sum;
+            cur_seg = s1.seg;
+            cur_sum = 0.f;
+          }
+          cur_sum += h1;
+        }
+      }
+      if (ok) {
+        seg_smem[cur_seg * BM + row] = cur_sum;
+        // Eq. 2: mean over the step's rows of mass(row, scale) / rowsum(row); rows past t_q are padding
+        const bool live = q0 + x * BM + row < p.t_q;
+        const float inv = live ? 1.f / l_sum : 0.f;
+        for (int s = 0; s <= p.step; ++s) {
+          float v = live ? seg_smem[s * BM + row] * inv : 0.f;
+#pragma unroll
+          for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
+          if (lane == 0) atomicAdd(acc_smem + s, v);
+        }
+      }
+    }
+  }
+
+  tc_fence_before();
+  __syncthreads();
+  if ((int)threadIdx.x <= p.step && *abort_flag == 0)
+    atomicAdd(p.beta_row + (int64_t)head * p.K * p.K + threadIdx.x, acc_smem[threadIdx.x] / (float)p.t_q);
+  if (warp == 0) {
+    tc_fence_after();
+    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem), "r"(TMEM_COLS) : "memory");
+  }
+}
+
+}  // namespace calib
+
+// ---------------------------------------------------------------------------------- host side
+struct CalibTcState {
+  PFN_cuTensorMapEncodeTiled_v12000 encode = nullptr;
+  std::vector<int2> host_descs;          // all steps, concatenated (kept alive for the upload)
+  std::vector<int> first, count;         // per step
+  const int2* dev_descs = nullptr;
+  bool ready = false;
+};
+
+uint64_t calib_tc_desc_bytes(const heatkv_config& cfg) {
+  uint64_t n = 0;
+  for (int step = 0; step < cfg.K; ++step)
+    for (int i = 0; i <= step; ++i) n += (uint64_t)(cfg.t[i] + calib::HALF - 1) / calib::HALF;
+  return n * sizeof(int2);
+}
+
+// `dev_table` is device memory of calib_tc_desc_bytes(cfg) bytes inside the context's metadata region.
+int calib_tc_create(const heatkv_config& cfg, void* dev_table, cudaStream_t stream, CalibTcState** out) {
+  *out = nullptr;
+  CalibTcState* st = new (std::nothrow) CalibTcState;
+  if (!st) return HEATKV_ERR_HOST_MEMORY;
+  *out = st;
+  if (cfg.d != calib::D || !dev_table) return HEATKV_OK;       // only head_dim 128 runs on this path
+  void* fn = nullptr;
+  cudaDriverEntryPointQueryResult qres;
+  if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &fn, cudaEnableDefault, &qres) != cudaSuccess ||
+      qres != cudaDriverEntryPointSuccess || !fn) {
+    cudaGetLastError();
+    return HEATKV_OK;
+  }
+  st->encode = reinterpret_cast<PFN_cuTensorMapEncodeTiled_v12000>(fn);
+  try {
+    for (int step = 0; step < cfg.K; ++step) {
+      st->first.push_back((int)st->host_descs.size());
+      int row0 = 0;
+      for (int i = 0; i <= step; ++i) {
+        for (int off = 0; off < cfg.t[i]; off += calib::HALF) {
+          int n = cfg.t[i] - off < calib::HALF ? cfg.t[i] - off : calib::HALF;
+          st->host_descs.push_back(make_int2(row0 + off, n | (i << 8)));
+        }
+        row0 += cfg.t[i];
+      }
+      st->count.push_back((int)st->host_descs.size() - st->first.back());
+    }
+  } catch (const std::bad_alloc&) {
+    return HEATKV_ERR_HOST_MEMORY;
+  }
+  if (cudaMemcpyAsync(dev_table, st->host_descs.data(), st->host_descs.size() * sizeof(int2), cudaMemcpyHostToDevice,
+                      stream) != cudaSuccess)
+    return HEATKV_ERR_CUDA;
+  // later calls may come on other streams: the table must be in place before create returns
+  if (cudaStreamSynchronize(stream) != cudaSuccess) return HEATKV_ERR_CUDA;
+  st->dev_descs = static_cast<const int2*>(dev_table);
+  if (cudaFuncSetAttribute(calib::calib_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)calib::SM_ALLOC) !=
+      cudaSuccess) {
+    cudaGetLastError();
+    return HEATKV_OK;
+  }
+  cudaFuncAttributes attr;
+  if (cudaFuncGetAttributes(&attr, calib::calib_tc_kernel) != cudaSuccess) {
+    cudaGetLastError();
+    return HEATKV_OK;
+  }
+  // the register hand-over inside the kernel must fit in what the launch really allocates
+  if (attr.numRegs * calib::THREADS < 128 * 72 + 256 * 216) return HEATKV_ERR_CUDA;
+  st->ready = true;
+  return HEATKV_OK;
+}
+
+void calib_tc_destroy(CalibTcState* st) { delete st; }
+
+bool calib_tc_supported(const CalibTcState* st, const AttnParams& p, int d, int n_seq) {
+  if (!st || !st->ready || d != calib::D || n_seq > 65535 || p.H > 65535) return false;
+  const int64_t s[6] = {p.q_seq, p.q_head, p.q_tok, p.kv_seq, p.kv_head, p.kv_tok};
+  for (int64_t v : s)
+    if (v & 7) return false;
+  return true;
+}
+
+namespace {
+bool encode_4d(CalibTcState* st, CUtensorMap* m, const void* base, int t, int H, int n_seq, int64_t s_tok, int64_t s_head,
+               int64_t s_seq) {
+  cuuint64_t dims[4] = {(cuuint64_t)calib::D, (cuuint64_t)t, (cuuint64_t)H, (cuuint64_t)n_seq};
+  auto fix = [](int64_t s) { return (cuuint64_t)((s > 0 ? s : 8) * 2); };
+  cuuint64_t strides[3] = {fix(s_tok), fix(s_head), fix(s_seq)};
+  cuuint32_t box[4] = {64, (cuuint32_t)calib::HALF, 1, 1};
+  cuuint32_t estr[4] = {1, 1, 1, 1};
+  return st->encode(m, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 4, const_cast<void*>(base), dims, strides, box, estr,
+                    CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                    CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+}  // namespace
+
+cudaError_t launch_calib_tc(CalibTcState* st, const AttnParams& p, int n_seq, cudaStream_t stream) {
+  calib::Maps maps;
+  if (!encode_4d(st, &maps.q, p.q, p.t_q, p.H, n_seq, p.q_tok, p.q_head, p.q_seq) ||
+      !encode_4d(st, &maps.k, p.k_new, p.n_own, p.H, n_seq, p.kv_tok, p.kv_head, p.kv_seq))
+    return cudaErrorInvalidValue;
+  dim3 grid((p.t_q + 2 * calib::BM - 1) / (2 * calib::BM), n_seq, p.H);
+  calib::calib_tc_kernel<<<grid, calib::THREADS, calib::SM_ALLOC, stream>>>(p, maps, st->dev_descs + st->first[p.step],
+                                                                            st->count[p.step]);
+  return cudaGetLastError();
+}
+
+}  // namespace heatkv

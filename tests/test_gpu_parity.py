@@ -169,10 +169,10 @@ def test_full_budget_equals_uncompressed(hk):
     _run_full_parity(hk, sh, ref, lambda ses: ses.schedule(scas=scores, b=1.0), hk.LAYOUT_PAGED)
 
 
-def _calibrate(hk, sh, seeds, bias=None, with_out=False):
+def _calibrate(hk, sh, seeds, bias=None, with_out=False, kernel=None):
     from paper_2605_14877_b200.sweep import Session
     sm = 1.0 / math.sqrt(sh.d)
-    ses = Session(sh.L, sh.H, sh.d, sh.t, sh.s, pool_rows=64, kernel=hk.KERNEL_GENERIC)
+    ses = Session(sh.L, sh.H, sh.d, sh.t, sh.s, pool_rows=64, kernel=hk.KERNEL_GENERIC if kernel is None else kernel)
     beta_dev = torch.zeros(sh.L, sh.H, sh.K, sh.K, dtype=torch.float32, device="cuda")
     bias_dev = None if bias is None else torch.from_numpy(bias).cuda()
     ref = np.zeros((sh.L, sh.H, sh.K, sh.K))
@@ -227,6 +227,22 @@ def test_calibration_mid_with_bias_and_output(hk):
     beta, scas, cas, ref = _calibrate(hk, sh, seeds=[5], bias=bias, with_out=True)
     mask = ref > 1e-5
     assert np.all(np.abs(beta - ref)[mask] <= RTOL_BETA * ref[mask])
+    assert np.allclose(beta.sum(axis=-1), 1.0, atol=2e-4)
+    for l in range(sh.L):
+        for h in range(sh.H):
+            assert np.allclose(scas[l, h], O.scas(ref[l, h], sh.s), rtol=RTOL_BETA, atol=1e-9)
+
+
+@pytest.mark.parametrize("with_bias", [False, True], ids=["plain", "bias"])
+def test_calibration_tensor_memory_kernel(hk, with_bias):
+    """Every step forced through the tcgen05 calibration kernel: one-row tiles, ragged source-scale
+    borders inside key tiles (36, 144, 400 tokens), an odd number of half-tiles, two query tiles."""
+    sh = W.Shape("mid", L=2, H=3, d=128, sides=W.SIDES_13[:11], n_seq=2, s=3)
+    bias = W.seg_bias_prior_lognormal(sh, 8) if with_bias else None
+    beta, scas, cas, ref = _calibrate(hk, sh, seeds=[5], bias=bias, kernel=hk.KERNEL_TCGEN05)
+    mask = ref > 1e-5
+    assert np.all(np.abs(beta - ref)[mask] <= RTOL_BETA * ref[mask]), float((np.abs(beta - ref)[mask] / ref[mask]).max())
+    assert np.all(np.triu(beta, 1) == 0)
     assert np.allclose(beta.sum(axis=-1), 1.0, atol=2e-4)
     for l in range(sh.L):
         for h in range(sh.H):
