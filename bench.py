@@ -198,6 +198,76 @@ def run_reference(args, rank):
     print(json.dumps(line), flush=True)
 
 
+def run_cache_workload(args):
+    """Cache-update kernels at a saturating shape (not the headline line): the larger-model layer shape
+    (32 heads, d=128, 16 sequences, one layer).  Appends are timed with every head storing (full
+    budget, paged and ragged); the in-place compaction of the ragged layout under a 1/5 budget.
+    Bytes are algorithmic: 8*d*t_k per storing head (K and V, read + write), 8*d*moved tokens per move."""
+    import paper_2605_14877_b200 as hk
+    from paper_2605_14877_b200.sweep import Session
+    torch.cuda.set_device(0)
+    sh = W.Shape("larger_layer", L=1, H=32, d=128, sides=W.SIDES_13, n_seq=16, s=3)
+    pk = peaks()
+    out = {"workload": "cache_update_saturating", "shape": {"H": sh.H, "d": sh.d, "n_seq": sh.n_seq, "scales": sh.K},
+           "peak_gbs": pk["hbm_gbs"], "peak_source": pk["source"]}
+    ks = [torch.randn(sh.n_seq, sh.H, sh.t[k], sh.d, device="cuda").to(torch.bfloat16) for k in range(sh.K)]
+    vs = [torch.randn_like(x) for x in ks]
+    flush = torch.empty(256 << 20, dtype=torch.uint8, device="cuda")
+    stream = torch.cuda.current_stream()
+    for name, layout, b in (("append_paged", hk.LAYOUT_PAGED, 1.0), ("append_ragged", hk.LAYOUT_RAGGED, 1.0),
+                            ("compact_ragged", hk.LAYOUT_RAGGED, 0.2)):
+        ses = Session(sh.L, sh.H, sh.d, sh.t, sh.s, pool_rows=sh.n_seq * sh.H * (sh.c[-2] + 64 * sh.K) + 64, layout=layout)
+        sch = ses.schedule(scas=W.synthetic_scas(sh, 0), b=b)
+        am, km, nk, _ = hk.heatkv_schedule_masks(sch, sh.K, sh.L, sh.H)
+        plan = hk.heatkv_schedule_plan(sch, layout)
+        ms = np.zeros(sh.K)
+        reps = max(3, min(args.steps, 10))
+        for rep in range(reps + 1):
+            ids = [hk.heatkv_seq_open(ses.ctx, sch) for _ in range(sh.n_seq)]
+            for step in range(sh.K - 1):
+                flush.fill_(step)
+                e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+                # compact_ragged: the eviction before the scale and the update after the layer (in-place
+                # compaction of G_k \\ A_k, then the append) are timed together
+                if name != "compact_ragged":
+                    ses.pre_step(ids, step)
+                e0.record(stream)
+                if name == "compact_ragged":
+                    ses.pre_step(ids, step)
+                hk.heatkv_append_compact(ses.ctx, ids, 0, step, ks[step], vs[step], None)
+                e1.record(stream)
+                torch.cuda.synchronize()
+                if rep > 0:
+                    ms[step] += e0.elapsed_time(e1) / reps
+            for i in ids:
+                hk.heatkv_seq_close(ses.ctx, i)
+        rows = []
+        hdr = plan[:20]
+        for step in range(sh.K - 1):
+            storing = sum(1 for h in range(sh.H) if (int(km[step, 0, h]) >> step) & 1)
+            nbytes = 8 * sh.d * sh.t[step] * storing * sh.n_seq
+            if name == "compact_ragged":
+                # plus the tokens moved by both evictions of the step: the plan's move lists (src, dst, n, 0)
+                off_move = int(hdr[10])
+                moved = 0
+                for off_b, off_c in ((int(hdr[11]), int(hdr[12])), (int(hdr[13]), int(hdr[14]))):
+                    for h in range(sh.H):
+                        u = (step * sh.L + 0) * sh.H + h
+                        b0, cnt = int(plan[off_b + u]), int(plan[off_c + u])
+                        for m in range(cnt):
+                            moved += int(plan[off_move + 4 * (b0 + m) + 2])
+                nbytes += 8 * sh.d * moved * sh.n_seq
+            if nbytes and ms[step] > 0:
+                rows.append({"scale": step + 1, "MB": round(nbytes / 1e6, 2), "us": round(ms[step] * 1e3, 2),
+                             **({"moved_tokens_per_seq": moved} if name == "compact_ragged" else {}),
+                             "GBs": round(nbytes / (ms[step] * 1e-3) / 1e9, 1),
+                             "frac": round(nbytes / (ms[step] * 1e-3) / 1e9 / pk["hbm_gbs"], 3)})
+        out[name] = rows
+        hk.heatkv_schedule_free(sch)
+        ses.close()
+    print(json.dumps(out), flush=True)
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -208,6 +278,8 @@ def main():
     ap.add_argument("--kernel", default="auto", choices=["auto", "generic", "tcgen05"])
     ap.add_argument("--launch", default="graph", choices=["graph", "eager"],
                     help="timed sweeps replay one captured CUDA graph of the 13-step sweep, or issue every call")
+    ap.add_argument("--workload", default="config2", choices=["config2", "cache"],
+                    help="config2: the headline line; cache: append / compaction GB/s at a saturating shape")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true", help="skip the host-buffer leg (profiling runs)")
     args = ap.parse_args()
@@ -218,6 +290,10 @@ def main():
     local = int(os.environ.get("LOCAL_RANK", "0"))
     if args.impl == "reference":
         run_reference(args, rank)
+        return
+    if args.workload == "cache":
+        if rank == 0:
+            run_cache_workload(args)
         return
 
     import paper_2605_14877_b200 as hk
