@@ -268,6 +268,93 @@ def run_cache_workload(args):
     print(json.dumps(out), flush=True)
 
 
+def run_model_workload(args, which):
+    """Whole-model sweeps (not the headline line).  `full`: 2B-class full model cache, 32 layers x 16
+    heads, batch 8, budgets 1/5, 1/10, 1/20.  `larger`: 40 layers x 32 heads, batch 16, 1/20.  `serving`:
+    64 concurrent images of the 2B shape, per-request budgets from {1/5, 1/10, 1/20, 1/40}, paged cache,
+    four admission waves one scale apart.  All layers reuse one layer's seeded activations (the kernels see
+    per-layer schedules, caches and biases); calls are issued one by one in generation order.
+    Attention + cache path only: images/s excludes everything else a model does."""
+    import paper_2605_14877_b200 as hk
+    from paper_2605_14877_b200.sweep import Session
+    torch.cuda.set_device(0)
+    sh = {"full": W.CFG3, "larger": W.CFG4, "serving": W.CFG5}[which]
+    scores = W.synthetic_scas(sh, 0)
+    bias_dev = torch.from_numpy(W.seg_bias_prior_lognormal(sh, 0)).cuda()
+    data = W.qkv_layer(sh, 0, 0, device="cuda")
+    out = torch.zeros_like(data[0])
+    cfg0 = hk.Config.make(sh.L, sh.H, sh.d, sh.t, sh.s)
+    results = []
+    runs = {"full": [[b] * sh.n_seq for b in (1 / 5, 1 / 10, 1 / 20)], "larger": [[1 / 20] * sh.n_seq],
+            "serving": [W.serving_budgets(sh.n_seq, 0)]}[which]
+    n_waves = 4 if which == "serving" else 1
+    wave = sh.n_seq // n_waves
+    for budgets in runs:
+        schs, rows = {}, {}
+        for b in sorted(set(budgets)):
+            schs[b] = hk.heatkv_build_schedule(cfg0, scas=scores, b=b)
+            rows[b] = hk.heatkv_schedule_footprint(schs[b], hk.LAYOUT_PAGED)[1]
+        pool_rows = sum(rows[b] for b in budgets) + 64
+        ses = Session(sh.L, sh.H, sh.d, sh.t, sh.s, pool_rows=pool_rows, meta_bytes=256 << 20)
+        stream = torch.cuda.current_stream()
+
+        def generation(measure):
+            ids = [None] * sh.n_seq
+            peak_used, peak_reserved = 0, 0
+            for tick in range(sh.K + n_waves - 1):
+                for w in range(n_waves):
+                    step = tick - w
+                    if step < 0 or step >= sh.K:
+                        continue
+                    members = list(range(w * wave, (w + 1) * wave))
+                    if step == 0:
+                        for s_ in members:
+                            ids[s_] = hk.heatkv_seq_open(ses.ctx, schs[budgets[s_]])
+                    wid = [ids[s_] for s_ in members]
+                    lo, hi = ses.step_slices(step)
+                    q, k, v = (x[members[0]: members[-1] + 1, :, lo:hi] for x in data)
+                    o = out[members[0]: members[-1] + 1, :, lo:hi]
+                    st = hk.Strides.of(q, k, o)
+                    ses.pre_step(wid, step)
+                    for l in range(sh.L):
+                        hk.heatkv_scale_attention(ses.ctx, wid, l, step, q, k, v, st, bias_dev[l, step], o)
+                        hk.heatkv_append_compact(ses.ctx, wid, l, step, k, v, st)
+                if measure:
+                    a = hk.heatkv_allocator_stats(ses.ctx)
+                    peak_used, peak_reserved = max(peak_used, a.used_tokens), max(peak_reserved, a.reserved_rows)
+            a = hk.heatkv_allocator_stats(ses.ctx)
+            for i in ids:
+                hk.heatkv_seq_close(ses.ctx, i)
+            return a, peak_used, peak_reserved
+
+        generation(False)
+        torch.cuda.synchronize()
+        reps = max(1, min(args.steps, 3))
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        t0 = time.perf_counter()
+        e0.record(stream)
+        for _ in range(reps):
+            a, peak_used, peak_reserved = generation(True)
+        e1.record(stream)
+        torch.cuda.synchronize()
+        ms = max(e0.elapsed_time(e1), 1e3 * (time.perf_counter() - t0)) / reps
+        assert hk.heatkv_device_status(ses.ctx) == 0
+        n_images = sh.n_seq / (2 if which != "serving" else 1)      # cond/uncond pair = one image outside serving
+        full_bytes = sh.n_seq * sh.L * sh.H * sh.c[-2] * sh.d * 4
+        results.append({"budgets": sorted(set(round(b, 4) for b in budgets)), "ms_per_generation": round(ms, 2),
+                        "images_per_s": round(n_images / (ms * 1e-3), 2),
+                        "cache_GB_end": round(a.used_tokens * sh.d * 4 / 1e9, 3),
+                        "cache_GB_uncompressed": round(full_bytes / 1e9, 3),
+                        "reserved_GB": round(a.reserved_rows * sh.d * 4 / 1e9, 3),
+                        "occupancy_end": round(a.used_tokens / max(a.reserved_rows, 1), 3),
+                        "peak_reserved_rows": int(peak_reserved), "pool_rows": int(a.pool_rows)})
+        for sch in schs.values():
+            hk.heatkv_schedule_free(sch)
+        ses.close()
+    print(json.dumps({"workload": sh.name, "L": sh.L, "H": sh.H, "n_seq": sh.n_seq, "launch": "eager",
+                      "data": "synthetic, one layer's activations reused by all layers", "runs": results}), flush=True)
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -278,8 +365,9 @@ def main():
     ap.add_argument("--kernel", default="auto", choices=["auto", "generic", "tcgen05"])
     ap.add_argument("--launch", default="graph", choices=["graph", "eager"],
                     help="timed sweeps replay one captured CUDA graph of the 13-step sweep, or issue every call")
-    ap.add_argument("--workload", default="config2", choices=["config2", "cache"],
-                    help="config2: the headline line; cache: append / compaction GB/s at a saturating shape")
+    ap.add_argument("--workload", default="config2", choices=["config2", "cache", "full", "larger", "serving"],
+                    help="config2: the headline line; cache: append / compaction GB/s at a saturating shape; "
+                         "full / larger / serving: whole-model sweeps of the other workloads")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true", help="skip the host-buffer leg (profiling runs)")
     args = ap.parse_args()
@@ -294,6 +382,10 @@ def main():
     if args.workload == "cache":
         if rank == 0:
             run_cache_workload(args)
+        return
+    if args.workload in ("full", "larger", "serving"):
+        if rank == 0:
+            run_model_workload(args, args.workload)
         return
 
     import paper_2605_14877_b200 as hk
