@@ -131,6 +131,33 @@ attn_tc_kernel(const __grid_constant__ AttnParams p, const __grid_constant__ Map
     asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
   }
   if (warp == 0) {
+    // The thread that initialised the barriers starts the first copies (both Q tiles, K and V of key
+    // tile 0) right away, so their latency runs under the TMEM allocation and the CTA-wide barrier.
+    if (threadIdx.x == 0) {
+      for (int x = 0; x < nq; ++x) {
+        mbar_expect_tx(bar(Q_FULL + x), TILE_BYTES);
+        for (int ch = 0; ch < 2; ++ch)
+          for (int hf = 0; hf < 2; ++hf)
+            tma_load_4d(sbase + SM_Q + x * TILE_BYTES + ch * HALF_COLS_BYTES + hf * SLOT_BYTES, &maps.q, ch * 64,
+                        q0 + x * BM + hf * HALF, head, seq, bar(Q_FULL + x));
+      }
+      Slot sl[2];
+      for (int hf = 0; hf < 2; ++hf) sl[hf] = get_slot(hf, descs, n_desc, n_slots, base_row, p.n_own, p.step);
+      mbar_expect_tx(bar(K_FULL + 0), TILE_BYTES);
+      for (int hf = 0; hf < 2; ++hf)
+        for (int ch = 0; ch < 2; ++ch) {
+          uint32_t dst = sbase + SM_K + ch * HALF_COLS_BYTES + hf * SLOT_BYTES;
+          if (sl[hf].pool_row >= 0) tma_load_2d(dst, &maps.k_pool, ch * 64, sl[hf].pool_row, bar(K_FULL + 0));
+          else tma_load_4d(dst, &maps.k_own, ch * 64, -sl[hf].pool_row - 1, head, seq, bar(K_FULL + 0));
+        }
+      mbar_expect_tx(bar(V_FULL + 0), TILE_BYTES);
+      for (int hf = 0; hf < 2; ++hf)
+        for (int ch = 0; ch < 2; ++ch) {
+          uint32_t dst = sbase + SM_V + ch * HALF_COLS_BYTES + hf * SLOT_BYTES;
+          if (sl[hf].pool_row >= 0) tma_load_2d(dst, &maps.v_pool, ch * 64, sl[hf].pool_row, bar(V_FULL + 0));
+          else tma_load_4d(dst, &maps.v_own, ch * 64, -sl[hf].pool_row - 1, head, seq, bar(V_FULL + 0));
+        }
+    }
     __syncwarp();
     asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(sbase + SM_TMEM_PTR), "r"(512u)
                  : "memory");
@@ -148,19 +175,10 @@ attn_tc_kernel(const __grid_constant__ AttnParams p, const __grid_constant__ Map
     // ------------------------------------------------------------------ TMA producer
     {
       const bool leader = elect_one();
-      uint32_t armed_k = 0, armed_v = 0;               // stage -> a copy was issued at least once
+      uint32_t armed_k = 1, armed_v = 1;               // stage -> a copy was issued at least once (tile 0: at CTA start)
       uint32_t par_k[KV_STAGES] = {0, 0}, par_v[KV_STAGES] = {0, 0};
-      if (leader) {
-        for (int x = 0; x < nq; ++x) {
-          mbar_expect_tx(bar(Q_FULL + x), TILE_BYTES);
-          for (int ch = 0; ch < 2; ++ch)
-            for (int hf = 0; hf < 2; ++hf)
-              tma_load_4d(sbase + SM_Q + x * TILE_BYTES + ch * HALF_COLS_BYTES + hf * SLOT_BYTES, &maps.q, ch * 64,
-                          q0 + x * BM + hf * HALF, head, seq, bar(Q_FULL + x));
-        }
-      }
       bool ok = true;
-      for (int j = 0; j < n_tiles && ok; ++j) {
+      for (int j = 1; j < n_tiles && ok; ++j) {
         const int st = j % KV_STAGES;
         const uint32_t use = (uint32_t)(j / KV_STAGES);
         Slot sl[2];
@@ -404,24 +422,36 @@ attn_tc_kernel(const __grid_constant__ AttnParams p, const __grid_constant__ Map
       if (ok) ok = __all_sync(0xffffffffu, mbar_wait(bar(PV_DONE + x), (n_tiles - 1) & 1, abort_flag, p.status));
       if (ok) {
         tc_fence_after();
+        // Normalise and round this row, park it in the shared memory of this tile's Q (no MMA reads it any
+        // more: every S product of the tile precedes the PV product just waited for), then let the warp
+        // write its 32 rows with two full 256-byte rows per store instruction.
         const float inv = 1.f / l_sum;
-        const bool live = q0 + x * BM + row < p.t_q;
-        __nv_bfloat16* dst = p.out + seq * p.o_seq + head * p.o_head + (int64_t)(q0 + x * BM + row) * p.o_tok;
+        unsigned char* stage = sgen + SM_Q + x * TILE_BYTES;     // [128 rows][16 chunks of 16 B], chunk ^ (row & 15)
 #pragma unroll
         for (int c = 0; c < 4; ++c) {
           uint32_t r[32];
           tmem_ld32(t_o + c * 32, r);
           tmem_wait_ld();
-          if (live) {
 #pragma unroll
-            for (int i = 0; i < 32; i += 8) {
-              int4 v;
-              v.x = (int)pack_bf16(__uint_as_float(r[i]) * inv, __uint_as_float(r[i + 1]) * inv);
-              v.y = (int)pack_bf16(__uint_as_float(r[i + 2]) * inv, __uint_as_float(r[i + 3]) * inv);
-              v.z = (int)pack_bf16(__uint_as_float(r[i + 4]) * inv, __uint_as_float(r[i + 5]) * inv);
-              v.w = (int)pack_bf16(__uint_as_float(r[i + 6]) * inv, __uint_as_float(r[i + 7]) * inv);
-              *reinterpret_cast<int4*>(dst + c * 32 + i) = v;
-            }
+          for (int i = 0; i < 32; i += 8) {
+            int4 v;
+            v.x = (int)pack_bf16(__uint_as_float(r[i]) * inv, __uint_as_float(r[i + 1]) * inv);
+            v.y = (int)pack_bf16(__uint_as_float(r[i + 2]) * inv, __uint_as_float(r[i + 3]) * inv);
+            v.z = (int)pack_bf16(__uint_as_float(r[i + 4]) * inv, __uint_as_float(r[i + 5]) * inv);
+            v.w = (int)pack_bf16(__uint_as_float(r[i + 6]) * inv, __uint_as_float(r[i + 7]) * inv);
+            const int chunk = c * 4 + (i >> 3);
+            *reinterpret_cast<int4*>(stage + row * 256 + ((chunk ^ (row & 15)) << 4)) = v;
+          }
+        }
+        __syncwarp();
+        const int row0 = (warp & 3) * 32;
+        __nv_bfloat16* dst = p.out + seq * p.o_seq + head * p.o_head + (int64_t)(q0 + x * BM) * p.o_tok;
+#pragma unroll 4
+        for (int k2 = 0; k2 < 16; ++k2) {
+          const int rr = row0 + 2 * k2 + (lane >> 4), chunk = lane & 15;
+          if (q0 + x * BM + rr < p.t_q) {
+            const int4 v = *reinterpret_cast<const int4*>(stage + rr * 256 + ((chunk ^ (rr & 15)) << 4));
+            *reinterpret_cast<int4*>(dst + (int64_t)rr * p.o_tok + chunk * 8) = v;
           }
         }
       }
