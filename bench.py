@@ -106,6 +106,21 @@ class ClockSampler:
                 "reasons": sorted(reasons), "samples": len(sm)}
 
 
+def aggregate_replicas(total_ms, e2e_ms, steps, dist=None, device="cpu", images_per_replica_step=1):
+    """Whole-job numbers of N independent replicas (the path has no exchange step): every rank times
+    its own K sweeps; the job's time is the slowest rank's, the job's work the sum over ranks.
+    Returns (ms_per_step, images/s, e2e images/s)."""
+    world = 1
+    if dist is not None:
+        tt = torch.tensor([total_ms, e2e_ms], dtype=torch.float64, device=device)
+        dist.all_reduce(tt, op=dist.ReduceOp.MAX)
+        total_ms, e2e_ms = (float(x) for x in tt.cpu())
+        world = dist.get_world_size()
+    images = images_per_replica_step * world
+    ms_per_step = total_ms / steps
+    return ms_per_step, images / (ms_per_step * 1e-3), images / (e2e_ms * 1e-3)
+
+
 def attention_flops(shape, am, n_seq):
     """Algorithmic flops of every (step) attention launch: 4*d*t_k*n_vis summed over (seq, head),
     n_vis = retained prior keys + the scale's own keys."""
@@ -550,13 +565,7 @@ def main():
         e2e_ms = max(e0.elapsed_time(e1), 1e3 * (time.perf_counter() - t0)) / e2e_steps
 
     # ---- aggregate over ranks (replicas): slowest rank's time
-    if dist is not None:
-        tt = torch.tensor([total_ms, e2e_ms], device=dev)
-        dist.all_reduce(tt, op=dist.ReduceOp.MAX)
-        total_ms, e2e_ms = (float(x) for x in tt.cpu())
-    images_per_step = 1 * world                     # one cond/uncond pair per replica
-    ms_per_step = total_ms / args.steps
-    value = images_per_step / (ms_per_step * 1e-3)
+    ms_per_step, value, e2e_value = aggregate_replicas(total_ms, e2e_ms, args.steps, dist, dev)   # one image pair per replica
 
     # ---- roofline of the dominant kernel: attn_tc_kernel (tcgen05), all its launches of a sweep
     pk = peaks()
@@ -589,7 +598,7 @@ def main():
                      "largest_launch": {"scale": big + 1, "tflops": flops[big] / (float(attn_ms[big]) * 1e-3) / 1e12,
                                         "frac": flops[big] / (float(attn_ms[big]) * 1e-3) / 1e12 / pk["bf16_tflops"]},
                      "traffic": TRAFFIC_BYTES_PER_SWEEP},
-        "e2e": {"value": images_per_step / (e2e_ms * 1e-3), "unit": UNIT, "h2d_bytes_per_step": h2d,
+        "e2e": {"value": e2e_value, "unit": UNIT, "h2d_bytes_per_step": h2d,
                 "d2h_bytes_per_step": d2h, "steps": e2e_steps},
         "gpu_launches": int(launches_per_sweep * args.steps),
         "clocks": clocks,
