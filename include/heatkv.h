@@ -82,8 +82,11 @@ typedef struct {
   int32_t kernel;                /* heatkv_kernel_choice                                    */
   float sm_scale;                /* logit scale; <= 0 selects 1/sqrt(d)                    */
   void* arena;                   /* DEVICE, caller-owned, 1024-byte aligned                */
-  uint64_t arena_bytes;          /* metadata region + K pool + V pool                      */
+  uint64_t arena_bytes;          /* metadata region + scratch region + K pool + V pool     */
   uint64_t meta_bytes;           /* bytes of the arena set aside for plans; 0 = default    */
+  uint64_t scratch_bytes;        /* bytes of the arena for partial results of heads whose key range is
+                                    split over several CTAs; 0 = default (1/8 of the arena, at most
+                                    128 MiB); too little only disables splitting                    */
 } heatkv_config;
 
 typedef struct {                 /* element strides of the [n_seq, H, t, d] activations    */
@@ -216,6 +219,15 @@ int heatkv_scale_attention(heatkv_ctx* ctx, const int* seq_ids /*HOST*/, int n_s
                            int step, const void* q, const void* k_new, const void* v_new,
                            const heatkv_strides* st, const float* seg_bias, void* out,
                            void* stream);
+
+/* How the tensor-memory attention kernel would cut the work of heatkv_scale_attention(seq_ids, layer,
+ * step): *split_tiles = longest run of 128-key tiles one CTA takes (0: every CTA takes a whole head's key
+ * range), *items = CTAs of the launch.  A head with more tiles than split_tiles is cut into equal pieces
+ * whose partial results meet in the arena's scratch region; the piece that arrives last merges them.  The
+ * choice minimises an estimate of the launch's makespan over the SMs and is cached per (schedule, step,
+ * layer, batch size).  Host only. */
+int heatkv_attention_split(heatkv_ctx* ctx, const int* seq_ids /*HOST*/, int n_seq, int layer, int step,
+                           int32_t* split_tiles, int32_t* items);
 
 /* Introspection (host state only unless noted). */
 int heatkv_cache_bytes(heatkv_ctx* ctx, int seq_id, uint64_t* actual, uint64_t* reserved);

@@ -1,5 +1,6 @@
 // C ABI of libheatkv: context, arena bookkeeping, sequence admission and the launch logic
 // of every entry point declared in heatkv.h.
+#include <algorithm>
 #include <cmath>
 #include <cstring>
 #include <map>
@@ -21,6 +22,7 @@ void tc_destroy(TcState* st);
 bool tc_supported(const TcState* st, const AttnParams& p, int d, int n_seq, bool calib);
 cudaError_t launch_attn_tc(TcState* st, const AttnParams& p, int d, int n_seq, bool calib, cudaStream_t stream,
                            int* launches);
+int tc_split_slot_floats();
 struct CalibTcState;
 uint64_t calib_tc_desc_bytes(const heatkv_config& cfg);
 int calib_tc_create(const heatkv_config& cfg, void* dev_table, cudaStream_t stream, CalibTcState** out);
@@ -112,6 +114,12 @@ struct heatkv_ctx {
   uint64_t launches = 0;
   TcState* tc = nullptr;
   CalibTcState* calib_tc = nullptr;
+  // key-range splitting of the tensor-memory attention kernel
+  float* split_partials = nullptr;
+  uint32_t* split_counters = nullptr;
+  uint64_t split_slots = 0, split_ctrs = 0;
+  int n_sm = 148;
+  std::map<uint64_t, int> split_choice;     // (plan uid, step, layer, n_seq) -> longest run of tiles per CTA (0: whole heads)
 };
 
 namespace {
@@ -228,6 +236,134 @@ int gather_seqs(heatkv_ctx* ctx, const int* seq_ids, int n_seq, int layer, int s
   return HEATKV_OK;
 }
 
+// ---- key-range splitting of the tensor-memory attention kernel -----------------------------------------
+// Items of one sequence under a longest run of `lmax` tiles (0: whole heads): count, partial slots, counters.
+struct SplitShape {
+  int items = 0, slots = 0, ctrs = 0;
+};
+
+SplitShape split_shape(const PlanEntry& pe, int step, int layer, int own_slots, int n_qp, int lmax) {
+  const Schedule& s = pe.sched;
+  const PlanHeader& h = pe.plan.header();
+  const int32_t* cnt = pe.plan.blob.data() + h.off_attn_cnt + s.at(step, layer, 0);
+  SplitShape r;
+  for (int hd = 0; hd < s.H; ++hd) {
+    const int tiles = (cnt[hd] + own_slots + 1) / 2;
+    const int ns = lmax > 0 ? (tiles + lmax - 1) / lmax : 1;
+    r.items += n_qp * ns;
+    if (ns > 1) { r.slots += n_qp * ns; r.ctrs += n_qp; }
+  }
+  return r;
+}
+
+// Estimated makespan (in units of one 128-key tile) of the launch when no CTA takes more than `lmax` tiles.
+// Items are handed to the SMs in dispatch order (heads by descending key count, pieces, query tile pairs,
+// sequences interleaved); for very large launches the list-scheduling bound total / SMs + longest is used.
+// The per-CTA constants were fitted to timings of launches with 2 to 32 (sequence, head) units.
+double split_makespan(const PlanEntry& pe, int step, int layer, int own_slots, int n_qp, int n_seq, int lmax, int n_sm) {
+  constexpr double FIXED = 6.0, PUBLISH = 1.5, MERGE_PER_PIECE = 1.5;
+  const Schedule& s = pe.sched;
+  const PlanHeader& h = pe.plan.header();
+  const int32_t* blob = pe.plan.blob.data();
+  const int32_t* cnt = blob + h.off_attn_cnt + s.at(step, layer, 0);
+  const int32_t* order = blob + h.off_order + s.at(step, layer, 0);
+  std::vector<double> costs;
+  double total = 0.0, longest = 0.0;
+  for (int i = 0; i < s.H; ++i) {
+    const int tiles = (cnt[order[i]] + own_slots + 1) / 2;
+    const int ns = lmax > 0 ? (tiles + lmax - 1) / lmax : 1;
+    const int piece = (tiles + ns - 1) / ns;
+    for (int pc = 0; pc < ns; ++pc) {
+      const int len = std::min(tiles, (pc + 1) * piece) - pc * piece;
+      const double c = len + FIXED + (ns > 1 ? PUBLISH + MERGE_PER_PIECE * (ns - 1) / ns : 0.0);
+      for (int q = 0; q < n_qp; ++q) costs.push_back(c);
+      total += c * n_qp;
+      longest = std::max(longest, c);
+    }
+  }
+  const size_t n_items = costs.size() * (size_t)n_seq;
+  if (n_items > 8192) return total * n_seq / n_sm + longest;
+  std::vector<double> sm(n_sm, 0.0);                       // binary min-heap of SM finish times
+  auto cmp = [](double a, double b) { return a > b; };
+  for (double c : costs)
+    for (int q = 0; q < n_seq; ++q) {
+      std::pop_heap(sm.begin(), sm.end(), cmp);
+      sm.back() += c;
+      std::push_heap(sm.begin(), sm.end(), cmp);
+    }
+  return *std::max_element(sm.begin(), sm.end());
+}
+
+// Fills the splitting fields of the launch parameters.  The choice is cached per (schedule, step, layer,
+// batch size); sequences of other schedules in the same call only raise the per-sequence bounds.
+void choose_split(heatkv_ctx* ctx, const int* seq_ids, int n_seq, int step, int layer, AttnParams* p) {
+  const int n_qp = (p->t_q + 255) / 256, own_slots = (p->n_own + HEATKV_PAGE_TOKENS - 1) / HEATKV_PAGE_TOKENS;
+  const PlanEntry& pe0 = *ctx->plans[ctx->seqs[seq_ids[0]].plan];
+  const uint64_t key = (pe0.uid << 24) ^ ((uint64_t)step << 20) ^ ((uint64_t)layer << 8) ^ (uint64_t)n_seq;
+  int lmax = 0;
+  auto it = ctx->split_choice.find(key);
+  if (it != ctx->split_choice.end()) {
+    lmax = it->second;
+  } else {
+    const Schedule& s = pe0.sched;
+    const int32_t* cnt = pe0.plan.blob.data() + pe0.plan.header().off_attn_cnt + s.at(step, layer, 0);
+    int max_tiles = 1;
+    for (int hd = 0; hd < s.H; ++hd) max_tiles = std::max(max_tiles, (cnt[hd] + own_slots + 1) / 2);
+    double best = split_makespan(pe0, step, layer, own_slots, n_qp, n_seq, 0, ctx->n_sm);
+    for (int div : {2, 3, 4, 6, 8, 12, 16}) {
+      const int cand = (max_tiles + div - 1) / div;
+      if (cand < 6) break;                                  // pieces about as short as the fixed cost never pay
+      const SplitShape sh = split_shape(pe0, step, layer, own_slots, n_qp, cand);
+      if ((uint64_t)sh.slots * n_seq > ctx->split_slots || (uint64_t)sh.ctrs * n_seq > ctx->split_ctrs) continue;
+      const double t = split_makespan(pe0, step, layer, own_slots, n_qp, n_seq, cand, ctx->n_sm);
+      if (t < 0.92 * best) { best = t; lmax = cand; }
+    }
+    ctx->split_choice[key] = lmax;
+  }
+  auto bounds = [&](int lm) {
+    SplitShape m;
+    int last_plan = -1;
+    for (int i = 0; i < n_seq; ++i) {
+      const int pi = ctx->seqs[seq_ids[i]].plan;
+      if (pi == last_plan) continue;
+      last_plan = pi;
+      const SplitShape sh = split_shape(*ctx->plans[pi], step, layer, own_slots, n_qp, lm);
+      m.items = std::max(m.items, sh.items); m.slots = std::max(m.slots, sh.slots); m.ctrs = std::max(m.ctrs, sh.ctrs);
+    }
+    return m;
+  };
+  SplitShape m = bounds(lmax);
+  if (lmax > 0 && ((uint64_t)m.slots * n_seq > ctx->split_slots || (uint64_t)m.ctrs * n_seq > ctx->split_ctrs)) {
+    lmax = 0;                                               // another schedule in the batch needs more scratch: whole heads
+    m = bounds(0);
+  }
+  // one plan for the whole call (the usual case): its heads, by descending key count, travel in the parameters
+  p->table_heads = 0;
+  bool one_plan = pe0.sched.H <= 64;
+  for (int i = 1; i < n_seq && one_plan; ++i) one_plan = ctx->seqs[seq_ids[i]].plan == ctx->seqs[seq_ids[0]].plan;
+  if (one_plan) {
+    const Schedule& s = pe0.sched;
+    const int32_t* blob = pe0.plan.blob.data();
+    const int32_t* cnt = blob + pe0.plan.header().off_attn_cnt + s.at(step, layer, 0);
+    const int32_t* order = blob + pe0.plan.header().off_order + s.at(step, layer, 0);
+    bool fits = true;
+    for (int i = 0; i < s.H; ++i) {
+      const int tiles = (cnt[order[i]] + own_slots + 1) / 2;
+      fits = fits && tiles <= 32767;
+      p->table_head[i] = (int16_t)order[i];
+      p->table_tiles[i] = (int16_t)tiles;
+    }
+    if (fits) p->table_heads = s.H;
+  }
+  p->n_seq = n_seq;
+  p->split_tiles = lmax;
+  p->items_per_seq = m.items;
+  p->slots_per_seq = m.slots;
+  p->ctrs_per_seq = m.ctrs;
+  p->split_partials = ctx->split_partials;
+  p->split_counters = ctx->split_counters;
+}
+
 }  // namespace
 
 extern "C" {
@@ -270,13 +406,30 @@ int heatkv_create(const heatkv_config* cfg, void* stream_, heatkv_ctx** out) {
   meta = (meta + 1023) / 1024 * 1024;
   if (meta < STATUS_BYTES + META_ALIGN || cfg->arena_bytes < meta + 2ull * HEATKV_PAGE_TOKENS * cfg->d * 2)
     return HEATKV_ERR_INVALID_ARG;
+  uint64_t scratch = cfg->scratch_bytes;
+  if (scratch == 0) scratch = std::min<uint64_t>(cfg->arena_bytes / 8, 128u << 20);
+  scratch = (scratch + 1023) / 1024 * 1024;
+  if (cfg->arena_bytes < meta + scratch + 2ull * HEATKV_PAGE_TOKENS * cfg->d * 2) return HEATKV_ERR_INVALID_ARG;
   const uint64_t row_bytes = (uint64_t)cfg->d * 2;
-  uint64_t rows = (cfg->arena_bytes - meta) / (2 * row_bytes);
+  uint64_t rows = (cfg->arena_bytes - meta - scratch) / (2 * row_bytes);
   rows = rows / HEATKV_PAGE_TOKENS * HEATKV_PAGE_TOKENS;
   if (rows > 0x7fffffffull) rows = 0x7fffffc0ull;
   ctx->meta = static_cast<unsigned char*>(cfg->arena);
   ctx->meta_bytes = meta;
-  ctx->k_pool = reinterpret_cast<__nv_bfloat16*>(ctx->meta + meta);
+  ctx->k_pool = reinterpret_cast<__nv_bfloat16*>(ctx->meta + meta + scratch);
+  {   // scratch region: arrival counters first (kept zero between launches), then the partial-result slots
+    const uint64_t ctr_bytes = std::min<uint64_t>(scratch / 4, 256u << 10) / 1024 * 1024;
+    const uint64_t slot_bytes = (uint64_t)tc_split_slot_floats() * 4;
+    ctx->split_counters = reinterpret_cast<uint32_t*>(ctx->meta + meta);
+    ctx->split_ctrs = ctr_bytes / 4;
+    ctx->split_partials = reinterpret_cast<float*>(ctx->meta + meta + ctr_bytes);
+    ctx->split_slots = (scratch - ctr_bytes) / slot_bytes;
+    if (ctr_bytes && cudaMemsetAsync(ctx->split_counters, 0, ctr_bytes, stream) != cudaSuccess) return HEATKV_ERR_CUDA;
+    int dev = 0, n_sm = 0;
+    if (cudaGetDevice(&dev) == cudaSuccess &&
+        cudaDeviceGetAttribute(&n_sm, cudaDevAttrMultiProcessorCount, dev) == cudaSuccess && n_sm > 0)
+      ctx->n_sm = n_sm;
+  }
   ctx->v_pool = ctx->k_pool + rows * cfg->d;
   ctx->pool_rows = rows;
   ctx->status = reinterpret_cast<uint32_t*>(ctx->meta);
@@ -451,6 +604,11 @@ int heatkv_scale_attention(heatkv_ctx* ctx, const int* seq_ids, int n_seq, int l
   cudaError_t e;
   if (use_tc) {
     int n = 0;
+    try {
+      choose_split(ctx, seq_ids, n_seq, step, layer, &p);
+    } catch (const std::bad_alloc&) {
+      return HEATKV_ERR_HOST_MEMORY;
+    }
     e = launch_attn_tc(ctx->tc, p, ctx->cfg.d, n_seq, false, stream, &n);
     ctx->launches += n;
   } else {
@@ -458,6 +616,25 @@ int heatkv_scale_attention(heatkv_ctx* ctx, const int* seq_ids, int n_seq, int l
     ctx->launches += 1;
   }
   return e == cudaSuccess ? HEATKV_OK : HEATKV_ERR_CUDA;
+}
+
+int heatkv_attention_split(heatkv_ctx* ctx, const int* seq_ids, int n_seq, int layer, int step, int32_t* split_tiles,
+                           int32_t* items) {
+  if (!ctx || !seq_ids || n_seq < 1 || n_seq > HEATKV_MAX_BATCH) return HEATKV_ERR_INVALID_ARG;
+  if (layer < 0 || layer >= ctx->cfg.L || step < 0 || step >= ctx->cfg.K) return HEATKV_ERR_INVALID_ARG;
+  for (int i = 0; i < n_seq; ++i)
+    if (!get_seq(ctx, seq_ids[i])) return HEATKV_ERR_INVALID_ARG;
+  AttnParams p;
+  std::memset(&p, 0, sizeof(p));
+  p.t_q = p.n_own = ctx->cfg.t[step];
+  try {
+    choose_split(ctx, seq_ids, n_seq, step, layer, &p);
+  } catch (const std::bad_alloc&) {
+    return HEATKV_ERR_HOST_MEMORY;
+  }
+  if (split_tiles) *split_tiles = p.split_tiles;
+  if (items) *items = p.items_per_seq * n_seq;
+  return HEATKV_OK;
 }
 
 int heatkv_calibrate_scores(heatkv_ctx* ctx, int layer, int step, int n_seq, const void* q, const void* k_full,

@@ -12,7 +12,9 @@
 //               so the result is exact).
 // TMEM columns: S_A/P_A 0..127, S_B/P_B 128..255, O_A 256..383, O_B 384..511.
 // The MMA order S_A S_B (PV_A S_A' PV_B S_B')* lets the softmax of one tile overlap the
-// tensor work of the other.  Every wait is bounded; on expiry the CTA records a status word,
+// tensor work of the other.  A launch is a list of work items (head, piece of the head's key range,
+// query tile pair); heads whose key range is longer than the launch's limit are cut into pieces whose
+// unnormalised results meet in a scratch region, where the piece that arrives last merges them.  Every wait is bounded; on expiry the CTA records a status word,
 // drains its own copies and leaves.
 #include "internal.h"
 #include "tc_common.cuh"
@@ -51,6 +53,11 @@ enum Bar : uint32_t {
 };
 constexpr uint32_t SM_TMEM_PTR = SM_BAR + N_BARS * 8;
 constexpr uint32_t SM_ABORT = SM_TMEM_PTR + 4;
+constexpr uint32_t SM_ITEM = SM_ABORT + 4;                     // int32[12]: the CTA's work item, decoded by warp 0
+// One partial result of a split head: unnormalised O of both query tiles (fp32, groups of four columns
+// outermost so that a warp's 32 rows touch consecutive 16-byte words), then the rows' running references
+// and row sums.
+constexpr int SPLIT_SLOT_FLOATS = 2 * BM * D + 2 * 2 * BM;
 
 
 struct Maps {
@@ -96,20 +103,79 @@ attn_tc_kernel(const __grid_constant__ AttnParams p, const __grid_constant__ Map
 
   // the shuffle makes the warp index provably warp-uniform, so role code stays on the uniform datapath
   const int warp = __shfl_sync(0xffffffffu, (int)(threadIdx.x >> 5), 0), lane = threadIdx.x & 31;
-  // grid = (query tile pairs, sequences, heads by descending key count): the heaviest heads of every
-  // sequence are dispatched first
-  const int seq = blockIdx.y;
-  const int q0 = blockIdx.x * (2 * BM);
-  const int nq = (q0 + BM < p.t_q) ? 2 : 1;          // does tile B hold any query?
-
+  // Work items.  grid.x = items_per_seq * n_seq, sequences interleaved.  The items of one sequence run
+  // over its heads by descending key count (the plan's order); a head whose key range exceeds
+  // split_tiles tiles is cut into equal pieces, and every (piece, query tile pair) is one item, pieces
+  // outermost.  Warp 0 finds this CTA's item with a prefix sum over the heads.
+  const int seq = blockIdx.x % p.n_seq;
+  const int item = blockIdx.x / p.n_seq;
   PlanView pv(p.seqs[seq].plan);
   const int u = (p.step * p.L + p.layer) * p.H;
-  const int head = pv.order()[u + blockIdx.z];
+  const int n_qp = (p.t_q + 2 * BM - 1) / (2 * BM);
+  volatile int32_t* item_smem = reinterpret_cast<volatile int32_t*>(sgen + SM_ITEM);
+  if (warp == 0) {
+    const int own_slots = (p.n_own + HALF - 1) / HALF;
+    if (lane == 0) item_smem[0] = -1;
+    __syncwarp();
+    int before = 0, slots_before = 0, ctrs_before = 0;
+    for (int base = 0; base < p.H; base += 32) {
+      const int i = base + lane;
+      int h = 0, tiles = 0, ns = 0, cnt = 0;
+      if (i < p.H) {
+        if (p.table_heads > 0) {                            // the host put the per-head table into the launch parameters
+          h = p.table_head[i];
+          tiles = p.table_tiles[i];
+        } else {
+          h = pv.order()[u + i];
+          tiles = (pv.attn_cnt()[u + h] + own_slots + 1) >> 1;
+        }
+        ns = p.split_tiles > 0 ? (tiles + p.split_tiles - 1) / p.split_tiles : 1;
+        cnt = n_qp * ns;
+      }
+      const int scnt = ns > 1 ? cnt : 0, ccnt = ns > 1 ? n_qp : 0;
+      int inc = cnt, sinc = scnt, cinc = ccnt;
+#pragma unroll
+      for (int o = 1; o < 32; o <<= 1) {
+        const int v0 = __shfl_up_sync(0xffffffffu, inc, o), v1 = __shfl_up_sync(0xffffffffu, sinc, o),
+                  v2 = __shfl_up_sync(0xffffffffu, cinc, o);
+        if (lane >= o) { inc += v0; sinc += v1; cinc += v2; }
+      }
+      const int excl = before + inc - cnt;
+      const bool mine = cnt > 0 && item >= excl && item < excl + cnt;
+      if (mine) {
+        item_smem[1] = tiles;
+        item_smem[2] = ns;
+        item_smem[3] = item - excl;                       // piece * n_qp + query tile pair
+        item_smem[4] = slots_before + sinc - scnt;        // first partial slot of this head
+        item_smem[5] = ctrs_before + cinc - ccnt;         // first arrival counter of this head
+        item_smem[0] = h;
+      }
+      const bool any = __any_sync(0xffffffffu, mine);
+      before += __shfl_sync(0xffffffffu, inc, 31);
+      slots_before += __shfl_sync(0xffffffffu, sinc, 31);
+      ctrs_before += __shfl_sync(0xffffffffu, cinc, 31);
+      if (any) break;
+    }
+  }
+  __syncthreads();
+  const int head = item_smem[0];
+  if (head < 0) return;                                   // padding item (sequences of a call may differ in item count)
+  const int n_split = item_smem[2];
+  const int piece = item_smem[3] / n_qp;
+  const int q0 = (item_smem[3] % n_qp) * (2 * BM);
+  const int slot_base = item_smem[4], ctr_base = item_smem[5];
+  const int nq = (q0 + BM < p.t_q) ? 2 : 1;          // does tile B hold any query?
   const int2* descs = pv.descs() + pv.attn_begin()[u + head];
   const int n_desc = pv.attn_cnt()[u + head];
   const int64_t base_row = p.seqs[seq].base_row;
   const int n_slots = n_desc + (p.n_own + HALF - 1) / HALF;
-  const int n_tiles = (n_slots + 1) / 2;
+  // this CTA's run of key tiles: [j0, j0 + n_tiles) of the head's ceil(n_slots / 2)
+  const int piece_tiles = (item_smem[1] + n_split - 1) / n_split;
+  const int j0 = piece * piece_tiles;
+  const int n_tiles = min(item_smem[1], j0 + piece_tiles) - j0;
+  // softmax state that outlives the role code (merging of split heads happens after it)
+  float m_ref = -INFINITY, l_sum = 0.f;
+  bool softmax_ok = false;
 
   if (threadIdx.x == 0) {
     *abort_flag = *reinterpret_cast<volatile uint32_t*>(p.status) != 0;   // an earlier CTA gave up: do not wait again
@@ -142,7 +208,7 @@ attn_tc_kernel(const __grid_constant__ AttnParams p, const __grid_constant__ Map
                         q0 + x * BM + hf * HALF, head, seq, bar(Q_FULL + x));
       }
       Slot sl[2];
-      for (int hf = 0; hf < 2; ++hf) sl[hf] = get_slot(hf, descs, n_desc, n_slots, base_row, p.n_own, p.step);
+      for (int hf = 0; hf < 2; ++hf) sl[hf] = get_slot(2 * j0 + hf, descs, n_desc, n_slots, base_row, p.n_own, p.step);
       mbar_expect_tx(bar(K_FULL + 0), TILE_BYTES);
       for (int hf = 0; hf < 2; ++hf)
         for (int ch = 0; ch < 2; ++ch) {
@@ -182,7 +248,7 @@ attn_tc_kernel(const __grid_constant__ AttnParams p, const __grid_constant__ Map
         const int st = j % KV_STAGES;
         const uint32_t use = (uint32_t)(j / KV_STAGES);
         Slot sl[2];
-        for (int hf = 0; hf < 2; ++hf) sl[hf] = get_slot(2 * j + hf, descs, n_desc, n_slots, base_row, p.n_own, p.step);
+        for (int hf = 0; hf < 2; ++hf) sl[hf] = get_slot(2 * (j0 + j) + hf, descs, n_desc, n_slots, base_row, p.n_own, p.step);
         // K first: the S product of the next tile needs it earliest
         if (use > 0) ok = warp_wait(bar(K_EMPTY + st), (use - 1) & 1, abort_flag, p.status);
         if (!ok) break;
@@ -312,11 +378,10 @@ attn_tc_kernel(const __grid_constant__ AttnParams p, const __grid_constant__ Map
       const uint32_t t_o = tmem + lane_base + 256 + x * 128;
       const float* bias_h = p.seg_bias ? p.seg_bias + head * p.K : nullptr;
       const float LOG2E = 1.4426950408889634f;
-      float m_ref = -INFINITY, l_sum = 0.f;
       bool ok = true;
       for (int j = 0; j < n_tiles && ok; ++j) {
-        Slot s0 = get_slot(2 * j, descs, n_desc, n_slots, base_row, p.n_own, p.step);
-        Slot s1 = get_slot(2 * j + 1, descs, n_desc, n_slots, base_row, p.n_own, p.step);
+        Slot s0 = get_slot(2 * (j0 + j), descs, n_desc, n_slots, base_row, p.n_own, p.step);
+        Slot s1 = get_slot(2 * (j0 + j) + 1, descs, n_desc, n_slots, base_row, p.n_own, p.step);
         const float b0 = bias_h ? bias_h[s0.seg] * LOG2E : 0.f;
         const float b1 = bias_h ? bias_h[s1.seg] * LOG2E : 0.f;
         ok = __all_sync(0xffffffffu, mbar_wait(bar(S_FULL + x), j & 1, abort_flag, p.status));
@@ -420,7 +485,26 @@ attn_tc_kernel(const __grid_constant__ AttnParams p, const __grid_constant__ Map
         mbar_arrive(bar(P_FULL + 2 * x + 1));
       }
       if (ok) ok = __all_sync(0xffffffffu, mbar_wait(bar(PV_DONE + x), (n_tiles - 1) & 1, abort_flag, p.status));
-      if (ok) {
+      softmax_ok = ok;
+      if (ok && n_split > 1) {
+        // A piece of a split head: publish the unnormalised O of this row with its reference and row sum.
+        tc_fence_after();
+        float* slot = p.split_partials +
+                      ((int64_t)seq * p.slots_per_seq + slot_base + item_smem[3]) * SPLIT_SLOT_FLOATS;
+        int4* ocol = reinterpret_cast<int4*>(slot) + x * BM + row;
+#pragma unroll
+        for (int c = 0; c < 4; ++c) {
+          uint32_t r[32];
+          tmem_ld32(t_o + c * 32, r);
+          tmem_wait_ld();
+#pragma unroll
+          for (int g = 0; g < 8; ++g)
+            ocol[(c * 8 + g) * (2 * BM)] = make_int4((int)r[4 * g], (int)r[4 * g + 1], (int)r[4 * g + 2], (int)r[4 * g + 3]);
+        }
+        slot[2 * BM * D + x * BM + row] = m_ref;
+        slot[2 * BM * D + 2 * BM + x * BM + row] = l_sum;
+        __threadfence();
+      } else if (ok) {
         tc_fence_after();
         // Normalise and round this row, park it in the shared memory of this tile's Q (no MMA reads it any
         // more: every S product of the tile precedes the PV product just waited for), then let the warp
@@ -460,6 +544,79 @@ attn_tc_kernel(const __grid_constant__ AttnParams p, const __grid_constant__ Map
 
   tc_fence_before();
   __syncthreads();
+  if (n_split > 1) {
+    // The piece that arrives last merges: sum over pieces of 2^(m_piece - m) * (O_piece, l_piece).
+    volatile int32_t* last_smem = item_smem + 8;
+    const int qp = item_smem[3] % n_qp;
+    if (threadIdx.x == 0) {
+      uint32_t* ctr = p.split_counters + (int64_t)seq * p.ctrs_per_seq + ctr_base + qp;
+      const uint32_t old = atomicAdd(ctr, 1u);
+      const bool last = old == (uint32_t)(n_split - 1);
+      if (last) *ctr = 0;                                     // ready for the next launch
+      last_smem[0] = last && *abort_flag == 0;
+    }
+    __syncthreads();
+    const int x = (warp - 4) >> 2;
+    if (last_smem[0] && warp >= 4 && x < nq && softmax_ok) {
+      __threadfence();
+      tc_fence_after();
+      const int row = (warp & 3) * 32 + lane;
+      const uint32_t t_o = tmem + ((uint32_t)((warp & 3) * 32) << 16) + 256 + x * 128;
+      const float* slots = p.split_partials + ((int64_t)seq * p.slots_per_seq + slot_base) * SPLIT_SLOT_FLOATS;
+      float m_all = m_ref;                                    // common reference and total row sum
+      for (int s2 = 0; s2 < n_split; ++s2) {
+        if (s2 == piece) continue;
+        const float* sl = slots + (int64_t)(s2 * n_qp + qp) * SPLIT_SLOT_FLOATS;
+        m_all = fmaxf(m_all, __ldcg(sl + 2 * BM * D + x * BM + row));
+      }
+      const float w_own = exp2f(m_ref - m_all);
+      float l_all = l_sum * w_own;
+      for (int s2 = 0; s2 < n_split; ++s2) {
+        if (s2 == piece) continue;
+        const float* sl = slots + (int64_t)(s2 * n_qp + qp) * SPLIT_SLOT_FLOATS;
+        l_all += __ldcg(sl + 2 * BM * D + 2 * BM + x * BM + row) * exp2f(__ldcg(sl + 2 * BM * D + x * BM + row) - m_all);
+      }
+      const float inv = 1.f / l_all;
+      const bool live = q0 + x * BM + row < p.t_q;
+      __nv_bfloat16* dst = p.out + seq * p.o_seq + head * p.o_head + (int64_t)(q0 + x * BM + row) * p.o_tok;
+#pragma unroll 1
+      for (int c = 0; c < 4; ++c) {
+        uint32_t r[32];
+        tmem_ld32(t_o + c * 32, r);
+        tmem_wait_ld();
+        float acc[32];
+#pragma unroll
+        for (int i = 0; i < 32; ++i) acc[i] = __uint_as_float(r[i]) * w_own;
+        for (int s2 = 0; s2 < n_split; ++s2) {
+          if (s2 == piece) continue;
+          const float* sl = slots + (int64_t)(s2 * n_qp + qp) * SPLIT_SLOT_FLOATS;
+          const float w = exp2f(__ldcg(sl + 2 * BM * D + x * BM + row) - m_all);
+          const float4* ocol = reinterpret_cast<const float4*>(sl) + (c * 8) * (2 * BM) + x * BM + row;
+#pragma unroll
+          for (int i = 0; i < 8; ++i) {
+            const float4 v = __ldcg(ocol + i * (2 * BM));
+            acc[4 * i] = fmaf(v.x, w, acc[4 * i]);
+            acc[4 * i + 1] = fmaf(v.y, w, acc[4 * i + 1]);
+            acc[4 * i + 2] = fmaf(v.z, w, acc[4 * i + 2]);
+            acc[4 * i + 3] = fmaf(v.w, w, acc[4 * i + 3]);
+          }
+        }
+        if (live) {
+#pragma unroll
+          for (int i = 0; i < 32; i += 8) {
+            int4 v;
+            v.x = (int)pack_bf16(acc[i] * inv, acc[i + 1] * inv);
+            v.y = (int)pack_bf16(acc[i + 2] * inv, acc[i + 3] * inv);
+            v.z = (int)pack_bf16(acc[i + 4] * inv, acc[i + 5] * inv);
+            v.w = (int)pack_bf16(acc[i + 6] * inv, acc[i + 7] * inv);
+            *reinterpret_cast<int4*>(dst + c * 32 + i) = v;
+          }
+        }
+      }
+    }
+    tc_fence_before();
+    __syncthreads();
+  }
   if (warp == 0) {
     tc_fence_after();
     asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem), "r"(512u) : "memory");
@@ -530,6 +687,8 @@ int tc_create(const heatkv_config& cfg, void* k_pool, void* v_pool, uint64_t poo
 
 void tc_destroy(TcState* st) { delete st; }
 
+int tc_split_slot_floats() { return tc::SPLIT_SLOT_FLOATS; }
+
 bool tc_supported(const TcState* st, const AttnParams& p, int d, int n_seq, bool calib) {
   if (!st || !st->ready || calib || d != tc::D || n_seq > 65535) return false;
   // TMA needs 16-byte aligned bases (checked by the caller) and strides that are multiples of 16 bytes
@@ -549,7 +708,8 @@ cudaError_t launch_attn_tc(TcState* st, const AttnParams& p, int d, int n_seq, b
       !encode_4d(st, &maps.k_own, p.k_new, p.n_own, p.H, n_seq, p.kv_tok, p.kv_head, p.kv_seq) ||
       !encode_4d(st, &maps.v_own, p.v_new, p.n_own, p.H, n_seq, p.kv_tok, p.kv_head, p.kv_seq))
     return cudaErrorInvalidValue;
-  dim3 grid((p.t_q + 2 * tc::BM - 1) / (2 * tc::BM), n_seq, p.H);
+  if (p.n_seq != n_seq || p.items_per_seq < 1) return cudaErrorInvalidValue;
+  dim3 grid((unsigned)p.items_per_seq * (unsigned)n_seq);
   tc::attn_tc_kernel<<<grid, tc::THREADS, tc::SM_ALLOC, stream>>>(p, maps);
   *launches = 1;
   return cudaGetLastError();

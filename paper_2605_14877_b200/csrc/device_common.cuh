@@ -35,6 +35,18 @@ struct AttnParams {
   uint32_t* status;               // device status word (non-zero = a bounded wait gave up)
   SeqRef seqs[HEATKV_MAX_BATCH];
   float* partials;                // calibration with a fixed summation order: per-warp partial masses, else null
+  // ---- key-range splitting of the tensor-memory attention kernel (split_tiles == 0: no splitting)
+  int32_t n_seq;                  // sequences of the call (work items interleave them)
+  int32_t split_tiles;            // longest run of 128-key tiles one CTA takes; a head with more is cut into pieces
+  int32_t items_per_seq;          // work items (head, piece, query tile pair) of one sequence, an upper bound
+  int32_t slots_per_seq;          // partial-result slots reserved per sequence
+  int32_t ctrs_per_seq;           // arrival counters reserved per sequence
+  int32_t table_heads;            // > 0: every sequence of the call follows one plan and the two tables below hold,
+                                  // for its heads by descending key count, the head index and its number of key tiles
+  int16_t table_head[64];
+  int16_t table_tiles[64];
+  float* split_partials;          // [n_seq * slots_per_seq][SPLIT_SLOT_FLOATS]
+  uint32_t* split_counters;       // [n_seq * ctrs_per_seq], zero between launches
 };
 
 struct CopyParams {

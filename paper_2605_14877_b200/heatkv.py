@@ -22,7 +22,7 @@ __all__ = [
     "heatkv_finalize_scores", "heatkv_build_schedule", "heatkv_schedule_free", "heatkv_schedule_masks", "heatkv_schedule_footprint",
     "heatkv_schedule_plan", "heatkv_seq_open", "heatkv_seq_close", "heatkv_append_compact", "heatkv_scale_attention",
     "heatkv_cache_bytes", "heatkv_retained_indices", "heatkv_export_head", "heatkv_allocator_stats",
-    "heatkv_launch_count", "heatkv_device_status", "heatkv_strerror", "arena_bytes_for",
+    "heatkv_launch_count", "heatkv_device_status", "heatkv_strerror", "heatkv_attention_split", "arena_bytes_for",
 ]
 
 MAX_K, MAX_BATCH, PAGE_TOKENS = 16, 128, 64
@@ -42,17 +42,18 @@ class Config(C.Structure):
     _fields_ = [("L", C.c_int32), ("H", C.c_int32), ("d", C.c_int32), ("K", C.c_int32),
                 ("t", C.c_int32 * MAX_K), ("s", C.c_int32), ("layout", C.c_int32), ("kernel", C.c_int32),
                 ("sm_scale", C.c_float), ("arena", C.c_void_p), ("arena_bytes", C.c_uint64),
-                ("meta_bytes", C.c_uint64)]
+                ("meta_bytes", C.c_uint64), ("scratch_bytes", C.c_uint64)]
 
     @classmethod
     def make(cls, L: int, H: int, d: int, t: Sequence[int], s: int, layout: int = LAYOUT_PAGED,
              kernel: int = KERNEL_AUTO, sm_scale: float = 0.0, arena: Optional[torch.Tensor] = None,
-             meta_bytes: int = 0) -> "Config":
+             meta_bytes: int = 0, scratch_bytes: int = 0) -> "Config":
         cfg = cls()
         cfg.L, cfg.H, cfg.d, cfg.K, cfg.s = L, H, d, len(t), s
         for i, v in enumerate(t):
             cfg.t[i] = int(v)
         cfg.layout, cfg.kernel, cfg.sm_scale, cfg.meta_bytes = layout, kernel, sm_scale, meta_bytes
+        cfg.scratch_bytes = scratch_bytes
         if arena is not None:
             cfg.arena = arena.data_ptr()
             cfg.arena_bytes = arena.numel() * arena.element_size()
@@ -90,7 +91,8 @@ def exported_symbols():
             "heatkv_build_schedule", "heatkv_schedule_free", "heatkv_schedule_masks",
             "heatkv_schedule_footprint", "heatkv_schedule_plan", "heatkv_seq_open", "heatkv_seq_close", "heatkv_append_compact",
             "heatkv_scale_attention", "heatkv_cache_bytes", "heatkv_retained_indices", "heatkv_export_head",
-            "heatkv_allocator_stats", "heatkv_launch_count", "heatkv_device_status", "heatkv_strerror"]
+            "heatkv_attention_split", "heatkv_allocator_stats", "heatkv_launch_count", "heatkv_device_status",
+            "heatkv_strerror"]
 
 
 def _load() -> C.CDLL:
@@ -120,6 +122,8 @@ _lib.heatkv_seq_close.argtypes = [_P, C.c_int]
 _lib.heatkv_append_compact.argtypes = [_P, C.POINTER(C.c_int), C.c_int, C.c_int, C.c_int, _P, _P, C.POINTER(Strides), _P]
 _lib.heatkv_scale_attention.argtypes = [_P, C.POINTER(C.c_int), C.c_int, C.c_int, C.c_int, _P, _P, _P,
                                         C.POINTER(Strides), _P, _P, _P]
+_lib.heatkv_attention_split.argtypes = [_P, C.POINTER(C.c_int), C.c_int, C.c_int, C.c_int, C.POINTER(C.c_int32),
+                                        C.POINTER(C.c_int32)]
 _lib.heatkv_cache_bytes.argtypes = [_P, C.c_int, C.POINTER(C.c_uint64), C.POINTER(C.c_uint64)]
 _lib.heatkv_retained_indices.argtypes = [_P, C.c_int, C.c_int, C.c_int, _P, C.POINTER(C.c_int)]
 _lib.heatkv_export_head.argtypes = [_P, C.c_int, C.c_int, C.c_int, _P, _P, _P]
@@ -160,10 +164,11 @@ def heatkv_strerror(status: int) -> str:
     return _lib.heatkv_strerror(int(status)).decode()
 
 
-def arena_bytes_for(pool_rows: int, d: int, meta_bytes: int = 1 << 24) -> int:
-    """Arena size that yields at least `pool_rows` rows in each of the K and V pools."""
+def arena_bytes_for(pool_rows: int, d: int, meta_bytes: int = 1 << 24, scratch_bytes: int = 1 << 26) -> int:
+    """Arena size that yields at least `pool_rows` rows in each of the K and V pools when the context is
+    created with the same (non-zero) `meta_bytes` and `scratch_bytes`."""
     rows = (pool_rows + PAGE_TOKENS - 1) // PAGE_TOKENS * PAGE_TOKENS
-    return (meta_bytes + 1023) // 1024 * 1024 + 2 * rows * d * 2
+    return (meta_bytes + 1023) // 1024 * 1024 + (scratch_bytes + 1023) // 1024 * 1024 + 2 * rows * d * 2
 
 
 def heatkv_create(cfg: Config, stream=None) -> int:
@@ -263,6 +268,14 @@ def heatkv_scale_attention(ctx, seq_ids, layer, step, q, k_new, v_new, strides, 
     st = C.byref(strides) if strides is not None else None
     _check(_lib.heatkv_scale_attention(ctx, ids, n, layer, step, _ptr(q), _ptr(k_new), _ptr(v_new), st,
                                        _ptr(seg_bias), _ptr(out), _stream(stream)), "heatkv_scale_attention")
+
+
+def heatkv_attention_split(ctx, seq_ids, layer, step):
+    """(longest run of 128-key tiles per CTA, 0 = whole heads; CTAs of the launch) for this attention call."""
+    ids, n = _ids(seq_ids)
+    a, b = C.c_int32(), C.c_int32()
+    _check(_lib.heatkv_attention_split(ctx, ids, n, layer, step, C.byref(a), C.byref(b)), "heatkv_attention_split")
+    return a.value, b.value
 
 
 def heatkv_cache_bytes(ctx: int, seq_id: int):

@@ -162,6 +162,34 @@ def test_tensor_memory_kernel_full_cache(hk):
                      kernel=hk.KERNEL_TCGEN05, check_cache=False)
 
 
+def test_key_range_splitting_is_used_and_exact(hk):
+    """Few heads with long key ranges: the launch cuts them into pieces that meet in the scratch region
+    (checked through heatkv_attention_split), and the merged outputs still match the oracle; a context
+    without scratch runs the same workload unsplit."""
+    from paper_2605_14877_b200.sweep import Session
+    sh = W.Shape("split", L=1, H=3, d=128, sides=W.SIDES_13[:12], n_seq=2, s=3)
+    scores = W.synthetic_scas(sh, 3)
+    ref = O.heatkv_schedule(scores, 0.6, sh.s, sh.sides)
+    bias = W.seg_bias_prior_lognormal(sh, 5)
+    with Session(sh.L, sh.H, sh.d, sh.t, sh.s, pool_rows=sh.n_seq * sh.H * (sh.c[-2] + 64 * sh.K)) as ses:
+        sch = ses.schedule(scas=scores, b=0.6)
+        ids = [hk.heatkv_seq_open(ses.ctx, sch) for _ in range(sh.n_seq)]
+        splits = [hk.heatkv_attention_split(ses.ctx, ids, 0, step) for step in range(sh.K)]
+        assert any(st > 0 for st, _ in splits[6:]), splits
+        assert all(items >= 1 for _, items in splits)
+        for i in ids:
+            hk.heatkv_seq_close(ses.ctx, i)
+        hk.heatkv_schedule_free(sch)
+    with Session(sh.L, sh.H, sh.d, sh.t, sh.s, pool_rows=4096, scratch_bytes=1024) as ses:
+        sch = ses.schedule(scas=scores, b=0.05)
+        sid = hk.heatkv_seq_open(ses.ctx, sch)
+        assert all(hk.heatkv_attention_split(ses.ctx, [sid], 0, step)[0] == 0 for step in range(sh.K))
+        hk.heatkv_seq_close(ses.ctx, sid)
+        hk.heatkv_schedule_free(sch)
+    _run_full_parity(hk, sh, ref, lambda ses: ses.schedule(scas=scores, b=0.6), hk.LAYOUT_PAGED, bias=bias,
+                     kernel=hk.KERNEL_AUTO)
+
+
 def test_full_budget_equals_uncompressed(hk):
     sh = W.Shape("full", L=1, H=2, d=64, sides=W.SIDES_13[:9], n_seq=1, s=2)
     scores = W.synthetic_scas(sh, 1)
