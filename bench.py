@@ -40,7 +40,7 @@ METRIC = "images_per_sec_scale_step_attention_2b_single_layer_20x"
 UNIT = "images/s"
 # dram__bytes_read.sum + dram__bytes_write.sum of the dominant kernel's launches of one sweep, from the ncu
 # capture summarised under profiles/; None once the kernel changed after the capture
-TRAFFIC_BYTES_PER_SWEEP = 304.2e6
+TRAFFIC_BYTES_PER_SWEEP = 311.8e6
 
 
 def peaks():
@@ -283,6 +283,53 @@ def run_cache_workload(args):
     print(json.dumps(out), flush=True)
 
 
+def run_few_heads_workload(args):
+    """Key-range splitting on launches that cannot fill the GPU with whole heads (not the headline line):
+    one sequence, 2 or 8 heads, d=128, 13 scales, full or half budget.  Every sweep is timed call by call
+    with the scratch region present (splitting allowed) and absent (whole heads only)."""
+    import paper_2605_14877_b200 as hk
+    from paper_2605_14877_b200.sweep import Session
+    torch.cuda.set_device(0)
+    rows = []
+    for H, b in ((2, 1.0), (8, 0.5)):
+        sh = W.Shape("few_heads", L=1, H=H, d=128, sides=W.SIDES_13, n_seq=1, s=3)
+        scores = W.synthetic_scas(sh, 0)
+        q, k, v = W.qkv_layer(sh, 0, 0, device="cuda")
+        c = [0] + sh.c
+        qs, ks, vs = ([x[:, :, c[i]:c[i + 1]].contiguous() for i in range(sh.K)] for x in (q, k, v))
+        outs = [torch.zeros_like(x) for x in qs]
+        flush = torch.empty(256 << 20, dtype=torch.uint8, device="cuda")
+        res = {"H": H, "budget": b}
+        for name, scratch in (("whole_heads_ms", 1024), ("split_ms", 1 << 27)):
+            ses = Session(sh.L, sh.H, sh.d, sh.t, sh.s, pool_rows=2 * sh.H * (sh.c[-2] + 64 * sh.K), scratch_bytes=scratch)
+            sch = ses.schedule(scas=scores, b=b)
+            ms, reps = np.zeros(sh.K), max(3, min(args.steps, 20))
+            for rep in range(reps + 2):
+                ids = [hk.heatkv_seq_open(ses.ctx, sch)]
+                if rep == 0 and scratch > 1024:
+                    res["split_tiles_per_scale"] = [hk.heatkv_attention_split(ses.ctx, ids, 0, st)[0] for st in range(sh.K)]
+                    res["ctas_per_scale"] = [hk.heatkv_attention_split(ses.ctx, ids, 0, st)[1] for st in range(sh.K)]
+                for step in range(sh.K):
+                    ses.pre_step(ids, step)
+                    flush.fill_(1)
+                    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+                    e0.record()
+                    hk.heatkv_scale_attention(ses.ctx, ids, 0, step, qs[step], ks[step], vs[step], None, None, outs[step])
+                    e1.record()
+                    hk.heatkv_append_compact(ses.ctx, ids, 0, step, ks[step], vs[step], None)
+                    torch.cuda.synchronize()
+                    if rep >= 2:
+                        ms[step] += e0.elapsed_time(e1) / reps
+                hk.heatkv_seq_close(ses.ctx, ids[0])
+            res[name] = [round(float(x), 4) for x in ms]
+            res[name.replace("_ms", "_sum_ms")] = round(float(ms.sum()), 4)
+            assert hk.heatkv_device_status(ses.ctx) == 0
+            hk.heatkv_schedule_free(sch)
+            ses.close()
+        rows.append(res)
+    print(json.dumps({"workload": "few_heads_key_range_splitting", "runs": rows}), flush=True)
+
+
 def run_model_workload(args, which):
     """Whole-model sweeps (not the headline line).  `full`: 2B-class full model cache, 32 layers x 16
     heads, batch 8, budgets 1/5, 1/10, 1/20.  `larger`: 40 layers x 32 heads, batch 16, 1/20.  `serving`:
@@ -380,9 +427,10 @@ def main():
     ap.add_argument("--kernel", default="auto", choices=["auto", "generic", "tcgen05"])
     ap.add_argument("--launch", default="graph", choices=["graph", "eager"],
                     help="timed sweeps replay one captured CUDA graph of the 13-step sweep, or issue every call")
-    ap.add_argument("--workload", default="config2", choices=["config2", "cache", "full", "larger", "serving"],
+    ap.add_argument("--workload", default="config2", choices=["config2", "cache", "full", "larger", "serving", "fewheads"],
                     help="config2: the headline line; cache: append / compaction GB/s at a saturating shape; "
-                         "full / larger / serving: whole-model sweeps of the other workloads")
+                         "full / larger / serving: whole-model sweeps of the other workloads; fewheads: key-range "
+                         "splitting on launches with few (sequence, head) units")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true", help="skip the host-buffer leg (profiling runs)")
     args = ap.parse_args()
@@ -397,6 +445,10 @@ def main():
     if args.workload == "cache":
         if rank == 0:
             run_cache_workload(args)
+        return
+    if args.workload == "fewheads":
+        if rank == 0:
+            run_few_heads_workload(args)
         return
     if args.workload in ("full", "larger", "serving"):
         if rank == 0:

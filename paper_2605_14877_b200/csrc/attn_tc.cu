@@ -29,6 +29,13 @@ constexpr int BN = 128;                 // keys per tile (two 64-row half-tiles)
 constexpr int HALF = 64;
 constexpr int THREADS = 384;
 constexpr int KV_STAGES = 2;
+// Registers are handed from the four utility warps to the eight softmax warps.  setmaxnreg only moves
+// registers inside the CTA's own allocation (threads x registers at launch), so the two budgets must fit
+// in it; an increase that cannot be served would block for ever.
+constexpr int REGS_LAUNCH = 168;        // what ptxas assigns under __launch_bounds__(384, 1)
+constexpr int REGS_SMALL = 72;
+constexpr int REGS_SOFTMAX = 216;
+static_assert(128 * REGS_SMALL + 256 * REGS_SOFTMAX <= THREADS * REGS_LAUNCH, "register hand-over exceeds the CTA's allocation");
 constexpr uint32_t HALF_COLS_BYTES = 128 * 128;        // one 64-column half of a 128-row tile: 16 KB
 constexpr uint32_t TILE_BYTES = 2 * HALF_COLS_BYTES;   // 32 KB
 constexpr uint32_t SLOT_BYTES = HALF * 128;            // 64 rows x 128 B inside one column half
@@ -236,7 +243,7 @@ attn_tc_kernel(const __grid_constant__ AttnParams p, const __grid_constant__ Map
 
   // register budget per warpgroup: 128*72 + 256*216 <= 64K
   if (warp < 4) {
-    reg_dealloc<72>();
+    reg_dealloc<REGS_SMALL>();
   if (warp == 0) {
     // ------------------------------------------------------------------ TMA producer
     {
@@ -368,7 +375,7 @@ attn_tc_kernel(const __grid_constant__ AttnParams p, const __grid_constant__ Map
     }
   }
   } else {
-    reg_alloc<216>();
+    reg_alloc<REGS_SOFTMAX>();
     // ------------------------------------------------------------------ softmax + epilogue
     const int x = (warp - 4) >> 2;                      // 0: tile A, 1: tile B
     if (x < nq) {
@@ -681,6 +688,13 @@ int tc_create(const heatkv_config& cfg, void* k_pool, void* v_pool, uint64_t poo
     cudaGetLastError();
     return HEATKV_OK;
   }
+  // the register hand-over inside the kernel must fit in what the launch really allocates
+  cudaFuncAttributes attr;
+  if (cudaFuncGetAttributes(&attr, tc::attn_tc_kernel) != cudaSuccess) {
+    cudaGetLastError();
+    return HEATKV_OK;
+  }
+  if (attr.numRegs * tc::THREADS < 128 * tc::REGS_SMALL + 256 * tc::REGS_SOFTMAX) return HEATKV_ERR_CUDA;
   st->ready = true;
   return HEATKV_OK;
 }
