@@ -330,6 +330,47 @@ def run_few_heads_workload(args):
     print(json.dumps({"workload": "few_heads_key_range_splitting", "runs": rows}), flush=True)
 
 
+def run_stability_workload(args):
+    """Synthetic analogue of the paper's S-CAS stability study (not the headline line): the S-CAS head
+    ordering is computed from 10 independently seeded calibration sets (4 sequences each) of a 4-layer x
+    16-head model with per-head log-normal locality, and the spread of every head's rank position across
+    the runs is reported per source scale, as the appendix does."""
+    import paper_2605_14877_b200 as hk
+    from paper_2605_14877_b200.analysis import scas_rank_dispersion
+    from paper_2605_14877_b200.sweep import Session
+    torch.cuda.set_device(0)
+    sh = W.Shape("stability", L=4, H=16, d=128, sides=W.SIDES_13, n_seq=2, s=3)
+    bias = torch.from_numpy(W.seg_bias_prior_lognormal(sh, 0)).cuda()
+    ses = Session(sh.L, sh.H, sh.d, sh.t, sh.s, pool_rows=64)
+    runs, n_runs, batches = [], 10, 2
+    ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    calib_ms = 0.0
+    for run in range(n_runs):
+        beta = torch.zeros(sh.L, sh.H, sh.K, sh.K, dtype=torch.float32, device="cuda")
+        for bt in range(batches):
+            for l in range(sh.L):
+                q, k, _ = W.qkv_layer(sh, 1000 + run * batches + bt, l, device="cuda")
+                ev0.record()
+                for step in range(sh.K):
+                    lo, hi = ses.step_slices(step)
+                    qs, ks = q[:, :, lo:hi], k[:, :, :hi]
+                    hk.heatkv_calibrate_scores(ses.ctx, l, step, sh.n_seq, qs, ks, None, hk.Strides.of(qs, ks),
+                                               bias[l, step], beta, None)
+                ev1.record()
+                torch.cuda.synchronize()
+                calib_ms += ev0.elapsed_time(ev1)
+        _, scas, _ = hk.heatkv_finalize_scores(ses.ctx, beta, batches * sh.n_seq, sh.L, sh.H, sh.K)
+        runs.append(scas)
+    assert hk.heatkv_device_status(ses.ctx) == 0
+    ses.close()
+    disp = scas_rank_dispersion(np.stack(runs), sh.s)
+    T = sh.L * sh.H
+    print(json.dumps({"workload": "scas_rank_stability", "heads": T, "runs": n_runs, "samples_per_run": batches * sh.n_seq,
+                      "rank_std_per_source_scale": {str(k + 1): round(float(disp[k]), 3) for k in range(sh.s, sh.K - 1)},
+                      "worst_fraction_of_ordering_range": round(float(disp.max()) / T, 4),
+                      "calibration_ms_total": round(calib_ms, 2)}), flush=True)
+
+
 def run_model_workload(args, which):
     """Whole-model sweeps (not the headline line).  `full`: 2B-class full model cache, 32 layers x 16
     heads, batch 8, budgets 1/5, 1/10, 1/20.  `larger`: 40 layers x 32 heads, batch 16, 1/20.  `serving`:
@@ -427,10 +468,11 @@ def main():
     ap.add_argument("--kernel", default="auto", choices=["auto", "generic", "tcgen05"])
     ap.add_argument("--launch", default="graph", choices=["graph", "eager"],
                     help="timed sweeps replay one captured CUDA graph of the 13-step sweep, or issue every call")
-    ap.add_argument("--workload", default="config2", choices=["config2", "cache", "full", "larger", "serving", "fewheads"],
+    ap.add_argument("--workload", default="config2", choices=["config2", "cache", "full", "larger", "serving", "fewheads", "stability"],
                     help="config2: the headline line; cache: append / compaction GB/s at a saturating shape; "
                          "full / larger / serving: whole-model sweeps of the other workloads; fewheads: key-range "
-                         "splitting on launches with few (sequence, head) units")
+                         "splitting on launches with few (sequence, head) units; stability: S-CAS rank spread "
+                         "over seeded calibration sets")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true", help="skip the host-buffer leg (profiling runs)")
     args = ap.parse_args()
@@ -445,6 +487,10 @@ def main():
     if args.workload == "cache":
         if rank == 0:
             run_cache_workload(args)
+        return
+    if args.workload == "stability":
+        if rank == 0:
+            run_stability_workload(args)
         return
     if args.workload == "fewheads":
         if rank == 0:

@@ -391,3 +391,29 @@ def kept_tokens_after_step(sch: Schedule, step: int) -> np.ndarray:
 def cache_bytes(kept: np.ndarray, d: int, dtype_bytes: int = 2) -> int:
     """sum over (layer, head) of kept_tokens * head_dim * 2 (K and V) * dtype bytes."""
     return int(kept.sum()) * d * 2 * dtype_bytes
+
+
+# ----------------------------------------------------------------------------- S-CAS stability (Appendix C)
+def scas_rank_dispersion(scas_runs: np.ndarray, s: int) -> np.ndarray:
+    """Stability of the S-CAS head ordering across calibration runs (Appendix, "S-CAS stability").
+
+    scas_runs: [R, L, H, K] S-CAS of R independent calibration sets.  For every prunable source scale
+    k in [s+1, K-1] each run orders the heads (order_from_scores); a head's rank position is recorded per
+    run, its standard deviation around the head's own mean rank is taken over the runs (population form,
+    1/R), and these are averaged over the heads.  Returns [K] (0 outside the prunable scales)."""
+    R, L, H, K = scas_runs.shape
+    T = L * H
+    out = np.zeros(K, dtype=np.float64)
+    for k in range(s + 1, K):
+        ranks = np.zeros((R, T), dtype=np.float64)
+        for r in range(R):
+            o = order_from_scores(np.asarray(scas_runs[r].reshape(T, K)[:, k - 1], dtype=np.float64))
+            for pos in range(T):
+                ranks[r, o[pos]] = pos
+        acc = 0.0
+        for head in range(T):
+            mean = sum(ranks[r, head] for r in range(R)) / R
+            var = sum((ranks[r, head] - mean) ** 2 for r in range(R)) / R
+            acc += var ** 0.5
+        out[k - 1] = acc / T
+    return out

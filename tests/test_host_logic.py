@@ -279,3 +279,11 @@ def test_paged_reservation_is_tighter_than_ragged_at_2b_shape(hk):
     B = O.budget_tokens(0.05, sh.L * sh.H, np.array(sh.c))
     assert peak_r == peak_p <= B
     assert rows_p < rows_r and rows_p < 1.35 * B
+
+
+def test_scas_rank_dispersion_matches_oracle():
+    from paper_2605_14877_b200.analysis import scas_rank_dispersion
+    rng = np.random.default_rng(3)
+    runs = rng.random((7, 3, 4, 9))
+    runs[2, 1, 2, 5] = runs[2, 0, 1, 5]                        # a tie: broken by head index on both sides
+    assert np.allclose(scas_rank_dispersion(runs, 3), O.scas_rank_dispersion(runs, 3), rtol=0, atol=1e-12)

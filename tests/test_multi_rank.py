@@ -27,7 +27,7 @@ def _worker(rank, world, port, out):
 
 def test_replica_aggregation_takes_slowest_rank_and_sums_work():
     world, port = 2, 29500 + os.getpid() % 2000
-    with mp.Manager() as m:
+    with mp.get_context("spawn").Manager() as m:
         out = m.dict()
         mp.spawn(_worker, args=(world, port, out), nprocs=world, join=True)
         res = [out[r] for r in range(world)]

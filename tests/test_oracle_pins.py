@@ -420,3 +420,23 @@ def test_workload_generator_is_seeded_and_sliceable():
     two = W.qkv_layer(W.TINY, 0, 0, n_seq=2)
     second = W.qkv_layer(W.TINY, 0, 0, n_seq=1, seq0=1)
     assert torch.equal(two[1][1], second[1][0])
+
+
+def test_scas_rank_dispersion_pins():
+    """Appendix on S-CAS stability: identical runs give zero dispersion; two runs that swap two adjacent
+    heads give those two heads a rank std of 1/2 each; scales outside the prunable range stay 0."""
+    rng = np.random.default_rng(0)
+    L, H, K, s = 2, 3, 6, 2
+    base = rng.random((L, H, K))
+    same = np.stack([base] * 4)
+    assert np.all(O.scas_rank_dispersion(same, s) == 0)
+    swapped = base.copy()
+    k = 3                                                    # 0-based source scale inside [s, K-2]
+    order = np.argsort(base.reshape(-1, K)[:, k], kind="stable")
+    a, b = order[1], order[2]
+    flat = swapped.reshape(-1, K)
+    flat[a, k], flat[b, k] = flat[b, k], flat[a, k]
+    d = O.scas_rank_dispersion(np.stack([base, swapped]), s)
+    assert np.isclose(d[k], 2 * 0.5 / (L * H))
+    assert np.all(d[:s] == 0) and d[K - 1] == 0
+    assert np.all(np.delete(d, k) == 0)
