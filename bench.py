@@ -376,7 +376,7 @@ def run_model_workload(args, which):
     heads, batch 8, budgets 1/5, 1/10, 1/20.  `larger`: 40 layers x 32 heads, batch 16, 1/20.  `serving`:
     64 concurrent images of the 2B shape, per-request budgets from {1/5, 1/10, 1/20, 1/40}, paged cache,
     four admission waves one scale apart.  All layers reuse one layer's seeded activations (the kernels see
-    per-layer schedules, caches and biases); calls are issued one by one in generation order.
+    per-layer schedules, caches and biases); one heatkv_attention_append call per (step, layer) in generation order.
     Attention + cache path only: images/s excludes everything else a model does."""
     import paper_2605_14877_b200 as hk
     from paper_2605_14877_b200.sweep import Session
@@ -420,8 +420,7 @@ def run_model_workload(args, which):
                     st = hk.Strides.of(q, k, o)
                     ses.pre_step(wid, step)
                     for l in range(sh.L):
-                        hk.heatkv_scale_attention(ses.ctx, wid, l, step, q, k, v, st, bias_dev[l, step], o)
-                        hk.heatkv_append_compact(ses.ctx, wid, l, step, k, v, st)
+                        hk.heatkv_attention_append(ses.ctx, wid, l, step, q, k, v, st, bias_dev[l, step], o)
                 if measure:
                     a = hk.heatkv_allocator_stats(ses.ctx)
                     peak_used, peak_reserved = max(peak_used, a.used_tokens), max(peak_reserved, a.reserved_rows)
@@ -468,6 +467,9 @@ def main():
     ap.add_argument("--kernel", default="auto", choices=["auto", "generic", "tcgen05"])
     ap.add_argument("--launch", default="graph", choices=["graph", "eager"],
                     help="timed sweeps replay one captured CUDA graph of the 13-step sweep, or issue every call")
+    ap.add_argument("--calls", default="fused", choices=["fused", "separate"],
+                    help="fused: heatkv_attention_append (one launch per step in the paged layout); separate: "
+                         "heatkv_scale_attention followed by heatkv_append_compact")
     ap.add_argument("--workload", default="config2", choices=["config2", "cache", "full", "larger", "serving", "fewheads", "stability"],
                     help="config2: the headline line; cache: append / compaction GB/s at a saturating shape; "
                          "full / larger / serving: whole-model sweeps of the other workloads; fewheads: key-range "
@@ -564,10 +566,14 @@ def main():
             ses.pre_step(ids, step)
             if events is not None and step in events:
                 events[step][0].record(stream)
-            hk.heatkv_scale_attention(ses.ctx, ids, 0, step, bq[step], bk[step], bv[step], None, bias[0, step], bo[step])
+            if args.calls == "fused":
+                hk.heatkv_attention_append(ses.ctx, ids, 0, step, bq[step], bk[step], bv[step], None, bias[0, step], bo[step])
+            else:
+                hk.heatkv_scale_attention(ses.ctx, ids, 0, step, bq[step], bk[step], bv[step], None, bias[0, step], bo[step])
             if events is not None and step in events:
                 events[step][1].record(stream)
-            hk.heatkv_append_compact(ses.ctx, ids, 0, step, bk[step], bv[step], None)
+            if args.calls != "fused":
+                hk.heatkv_append_compact(ses.ctx, ids, 0, step, bk[step], bv[step], None)
         for i in ids:
             hk.heatkv_seq_close(ses.ctx, i)
 
@@ -645,8 +651,11 @@ def main():
                 for src, dst in ((hq, dq), (hkk, dk), (hv, dv)):
                     dst[step].copy_(src[step], non_blocking=True)
                 ses.pre_step(ids, step)
-                hk.heatkv_scale_attention(ses.ctx, ids, 0, step, dq[step], dk[step], dv[step], None, bias[0, step], do[step])
-                hk.heatkv_append_compact(ses.ctx, ids, 0, step, dk[step], dv[step], None)
+                if args.calls == "fused":
+                    hk.heatkv_attention_append(ses.ctx, ids, 0, step, dq[step], dk[step], dv[step], None, bias[0, step], do[step])
+                else:
+                    hk.heatkv_scale_attention(ses.ctx, ids, 0, step, dq[step], dk[step], dv[step], None, bias[0, step], do[step])
+                    hk.heatkv_append_compact(ses.ctx, ids, 0, step, dk[step], dv[step], None)
                 hout[step].copy_(do[step], non_blocking=True)
             for i in ids:
                 hk.heatkv_seq_close(ses.ctx, i)
@@ -679,7 +688,7 @@ def main():
         "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
         "config": {"workload": shape.name, "L": shape.L, "H": shape.H, "d": shape.d, "scales": shape.K,
                    "tokens": shape.n_tokens, "n_seq": n_seq, "budget": B_BUDGET, "policy": "heatkv", "s": shape.s,
-                   "layout": args.layout, "kernel": args.kernel, "launch": args.launch,
+                   "layout": args.layout, "kernel": args.kernel, "launch": args.launch, "calls": args.calls,
                    "l2": "256 MB flush write between timed steps",
                    "one_image": "cond/uncond pair through one layer; x32 layers for a 2B-class model",
                    "n_k": [int(x) for x in nk], "replicas": world},

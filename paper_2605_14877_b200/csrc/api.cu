@@ -575,9 +575,12 @@ int heatkv_seq_close(heatkv_ctx* ctx, int seq_id) {
   return HEATKV_OK;
 }
 
-int heatkv_scale_attention(heatkv_ctx* ctx, const int* seq_ids, int n_seq, int layer, int step, const void* q,
-                           const void* k_new, const void* v_new, const heatkv_strides* st, const float* seg_bias,
-                           void* out, void* stream_) {
+// Attention of one layer at one step; with `with_update` the cache update after the layer follows: inside the
+// same launch in the paged layout (the plan never puts the new scale on a page this step still reads), as
+// the separate kernels otherwise.
+static int attention_impl(heatkv_ctx* ctx, const int* seq_ids, int n_seq, int layer, int step, const void* q,
+                          const void* k_new, const void* v_new, const heatkv_strides* st, const float* seg_bias,
+                          void* out, void* stream_, bool with_update) {
   if (!ctx || !q || !k_new || !v_new || !out) return HEATKV_ERR_INVALID_ARG;
   if (!aligned16(q) || !aligned16(k_new) || !aligned16(v_new) || !aligned16(out)) return HEATKV_ERR_INVALID_ARG;
   cudaStream_t stream = static_cast<cudaStream_t>(stream_);
@@ -597,6 +600,21 @@ int heatkv_scale_attention(heatkv_ctx* ctx, const int* seq_ids, int n_seq, int l
   p.t_q = p.n_own = ctx->cfg.t[step];
   p.step = step;
   p.layer = layer;
+  const bool stores = step + 1 < ctx->cfg.K;                  // the last scale is never cached
+  bool fuse = with_update && stores && ctx->cfg.layout == HEATKV_LAYOUT_PAGED;
+  if (fuse) {
+    // The append rides on the attention launch only while it is small (a launch-bound copy): its CTAs share
+    // the attention kernel's one-CTA-per-SM footprint, so a bandwidth-sized append keeps its own kernel.
+    constexpr uint64_t FUSE_LIMIT_BYTES = 8u << 20;
+    uint64_t storing = 0;
+    for (int i = 0; i < n_seq; ++i) {
+      const PlanEntry& pe = *ctx->plans[ctx->seqs[seq_ids[i]].plan];
+      const int32_t* cnt = pe.plan.blob.data() + pe.plan.header().off_app_cnt + pe.sched.at(step, layer, 0);
+      for (int hd = 0; hd < pe.sched.H; ++hd) storing += cnt[hd] > 0;
+    }
+    fuse = storing * (uint64_t)ctx->cfg.t[step] * ctx->cfg.d * 8 <= FUSE_LIMIT_BYTES;
+  }
+  if (fuse) p.append_tiles = (ctx->cfg.t[step] + HEATKV_PAGE_TOKENS - 1) / HEATKV_PAGE_TOKENS + 1;
   const int choice = ctx->cfg.kernel;
   bool use_tc = choice != HEATKV_KERNEL_GENERIC && tc_supported(ctx->tc, p, ctx->cfg.d, n_seq, false);
   if (choice == HEATKV_KERNEL_AUTO && p.t_q < 256) use_tc = false;
@@ -615,7 +633,25 @@ int heatkv_scale_attention(heatkv_ctx* ctx, const int* seq_ids, int n_seq, int l
     e = launch_attn_generic(p, ctx->cfg.d, n_seq, false, stream);
     ctx->launches += 1;
   }
-  return e == cudaSuccess ? HEATKV_OK : HEATKV_ERR_CUDA;
+  if (e != cudaSuccess) return HEATKV_ERR_CUDA;
+  if (!with_update) return HEATKV_OK;
+  if (fuse || !stores) {
+    for (int i = 0; i < n_seq; ++i) ctx->seqs[seq_ids[i]].done_step[layer] = (int16_t)step;
+    return HEATKV_OK;
+  }
+  return heatkv_append_compact(ctx, seq_ids, n_seq, layer, step, k_new, v_new, st, stream_);
+}
+
+int heatkv_scale_attention(heatkv_ctx* ctx, const int* seq_ids, int n_seq, int layer, int step, const void* q,
+                           const void* k_new, const void* v_new, const heatkv_strides* st, const float* seg_bias,
+                           void* out, void* stream_) {
+  return attention_impl(ctx, seq_ids, n_seq, layer, step, q, k_new, v_new, st, seg_bias, out, stream_, false);
+}
+
+int heatkv_attention_append(heatkv_ctx* ctx, const int* seq_ids, int n_seq, int layer, int step, const void* q,
+                            const void* k_new, const void* v_new, const heatkv_strides* st, const float* seg_bias,
+                            void* out, void* stream_) {
+  return attention_impl(ctx, seq_ids, n_seq, layer, step, q, k_new, v_new, st, seg_bias, out, stream_, true);
 }
 
 int heatkv_attention_split(heatkv_ctx* ctx, const int* seq_ids, int n_seq, int layer, int step, int32_t* split_tiles,

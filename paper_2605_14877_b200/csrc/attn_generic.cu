@@ -7,7 +7,7 @@
 // from k_new.  In calibration mode (Eq. 2) every key comes from k_full and the per-row
 // probability mass of every source scale is accumulated next to the online softmax, so the
 // attention matrix alpha is never formed.
-#include "device_common.cuh"
+#include "append_device.cuh"
 
 namespace heatkv {
 
@@ -63,6 +63,15 @@ __global__ void __launch_bounds__(GTHREADS, 2) attn_generic_kernel(const __grid_
   const int g = lane >> 2, qd = lane & 3;
   // attention: grid = (query tiles, sequences, heads by descending key count), so the heaviest heads of
   // every sequence are dispatched first; calibration: grid = (query tiles, heads, sequences)
+  if (!CALIB && (int)blockIdx.x >= (p.t_q + GM - 1) / GM) {
+    // cache update riding on this launch: one CTA per (destination half-tile, sequence, head)
+    const int sq = blockIdx.y, hd = blockIdx.z, j = blockIdx.x - (p.t_q + GM - 1) / GM;
+    const int64_t src = sq * p.kv_seq + hd * p.kv_head;
+    append_half_tile(p.seqs[sq].plan, p.seqs[sq].base_row, (p.step * p.L + p.layer) * p.H + hd, j, p.k_new + src,
+                     p.v_new + src, p.kv_tok, const_cast<__nv_bfloat16*>(p.k_pool), const_cast<__nv_bfloat16*>(p.v_pool),
+                     D, threadIdx.x, GTHREADS);
+    return;
+  }
   const int seq = CALIB ? blockIdx.z : blockIdx.y;
   const int q0 = blockIdx.x * GM;
   int head = CALIB ? blockIdx.y : blockIdx.z;
@@ -372,7 +381,7 @@ static cudaError_t launch_one(const AttnParams& p, int n_seq, cudaStream_t strea
     if (e != cudaSuccess) return e;
     configured = true;
   }
-  dim3 grid((p.t_q + GM - 1) / GM, CALIB ? p.H : n_seq, CALIB ? n_seq : p.H);
+  dim3 grid((p.t_q + GM - 1) / GM + (CALIB ? 0 : p.append_tiles), CALIB ? p.H : n_seq, CALIB ? n_seq : p.H);
   kern<<<grid, GTHREADS, GenericSmem<D>::BYTES, stream>>>(p);
   return cudaGetLastError();
 }

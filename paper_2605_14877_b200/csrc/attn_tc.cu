@@ -16,6 +16,7 @@
 // query tile pair); heads whose key range is longer than the launch's limit are cut into pieces whose
 // unnormalised results meet in a scratch region, where the piece that arrives last merges them.  Every wait is bounded; on expiry the CTA records a status word,
 // drains its own copies and leaves.
+#include "append_device.cuh"
 #include "internal.h"
 #include "tc_common.cuh"
 
@@ -114,6 +115,16 @@ attn_tc_kernel(const __grid_constant__ AttnParams p, const __grid_constant__ Map
   // over its heads by descending key count (the plan's order); a head whose key range exceeds
   // split_tiles tiles is cut into equal pieces, and every (piece, query tile pair) is one item, pieces
   // outermost.  Warp 0 finds this CTA's item with a prefix sum over the heads.
+  if ((int)blockIdx.x >= p.items_per_seq * p.n_seq) {
+    // cache update riding on this launch: one CTA per (destination half-tile, head, sequence)
+    const int idx = blockIdx.x - p.items_per_seq * p.n_seq;
+    const int sq = idx % p.n_seq, hd = (idx / p.n_seq) % p.H, j = idx / (p.n_seq * p.H);
+    const int64_t src = sq * p.kv_seq + hd * p.kv_head;
+    append_half_tile(p.seqs[sq].plan, p.seqs[sq].base_row, (p.step * p.L + p.layer) * p.H + hd, j, p.k_new + src,
+                     p.v_new + src, p.kv_tok, const_cast<__nv_bfloat16*>(p.k_pool), const_cast<__nv_bfloat16*>(p.v_pool),
+                     D, threadIdx.x, THREADS);
+    return;
+  }
   const int seq = blockIdx.x % p.n_seq;
   const int item = blockIdx.x / p.n_seq;
   PlanView pv(p.seqs[seq].plan);
@@ -723,7 +734,7 @@ cudaError_t launch_attn_tc(TcState* st, const AttnParams& p, int d, int n_seq, b
       !encode_4d(st, &maps.v_own, p.v_new, p.n_own, p.H, n_seq, p.kv_tok, p.kv_head, p.kv_seq))
     return cudaErrorInvalidValue;
   if (p.n_seq != n_seq || p.items_per_seq < 1) return cudaErrorInvalidValue;
-  dim3 grid((unsigned)p.items_per_seq * (unsigned)n_seq);
+  dim3 grid((unsigned)p.items_per_seq * (unsigned)n_seq + (unsigned)p.append_tiles * (unsigned)p.H * (unsigned)n_seq);
   tc::attn_tc_kernel<<<grid, tc::THREADS, tc::SM_ALLOC, stream>>>(p, maps);
   *launches = 1;
   return cudaGetLastError();

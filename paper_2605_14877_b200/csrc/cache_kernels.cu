@@ -1,54 +1,21 @@
 // Cache update kernels (Sec. 3.3): append of a new scale's K/V into the rows the plan
 // assigns, and the in-place left compaction of the ragged layout after an eviction.
 // Both are pure byte movers: 16-byte vector loads and stores, rows copied verbatim.
-#include "device_common.cuh"
+#include "append_device.cuh"
 
 namespace heatkv {
 
 constexpr int CP_THREADS = 128;
-constexpr int CP_UNROLL = 4;
 
 // ---------------------------------------------------------------- append
 // grid = (destination half-tile, head, sequence).  Destination half-tile j of a storing head
 // receives the next n_valid tokens of the step's K and V.
 __global__ void __launch_bounds__(CP_THREADS) append_kernel(const __grid_constant__ CopyParams p) {
   const int seq = blockIdx.z, head = blockIdx.y, j = blockIdx.x;
-  PlanView pv(p.seqs[seq].plan);
   const int u = (p.step * p.L + p.layer) * p.H + head;
-  const int cnt = pv.app_cnt()[u];
-  if (j >= cnt) return;
-  const int2* descs = pv.descs() + pv.app_begin()[u];
-  int tok0 = 0;
-  for (int i = 0; i < j; ++i) tok0 += descs[i].y & 0xff;
-  const int2 dsc = descs[j];
-  const int n = dsc.y & 0xff;
-  const int64_t row = p.seqs[seq].base_row + dsc.x;
-  const int ch_per_row = p.d / 8;
-  const int total = n * ch_per_row;                      // 16-byte chunks per tensor
-  const int64_t src_off = seq * p.kv_seq + head * p.kv_head + (int64_t)tok0 * p.kv_tok;
-  for (int base = threadIdx.x; base < total; base += CP_THREADS * CP_UNROLL) {
-    int4 kv[CP_UNROLL], vv[CP_UNROLL];
-#pragma unroll
-    for (int uu = 0; uu < CP_UNROLL; ++uu) {
-      int i = base + uu * CP_THREADS;
-      if (i < total) {
-        int r = i / ch_per_row, ch = i % ch_per_row;
-        int64_t off = src_off + (int64_t)r * p.kv_tok + ch * 8;
-        kv[uu] = __ldg(reinterpret_cast<const int4*>(p.k_new + off));
-        vv[uu] = __ldg(reinterpret_cast<const int4*>(p.v_new + off));
-      }
-    }
-#pragma unroll
-    for (int uu = 0; uu < CP_UNROLL; ++uu) {
-      int i = base + uu * CP_THREADS;
-      if (i < total) {
-        int r = i / ch_per_row, ch = i % ch_per_row;
-        int64_t off = (row + r) * p.d + ch * 8;
-        *reinterpret_cast<int4*>(p.k_pool + off) = kv[uu];
-        *reinterpret_cast<int4*>(p.v_pool + off) = vv[uu];
-      }
-    }
-  }
+  const int64_t src = seq * p.kv_seq + head * p.kv_head;
+  append_half_tile(p.seqs[seq].plan, p.seqs[seq].base_row, u, j, p.k_new + src, p.v_new + src, p.kv_tok, p.k_pool,
+                   p.v_pool, p.d, threadIdx.x, CP_THREADS);
 }
 
 // ---------------------------------------------------------------- in-place compaction

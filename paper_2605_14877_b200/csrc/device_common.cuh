@@ -45,6 +45,8 @@ struct AttnParams {
                                   // for its heads by descending key count, the head index and its number of key tiles
   int16_t table_head[64];
   int16_t table_tiles[64];
+  int32_t append_tiles;           // > 0: the launch also stores the step's K/V (paged layout): that many destination
+                                  // half-tile slots per (sequence, head) run as extra CTAs after the attention CTAs
   float* split_partials;          // [n_seq * slots_per_seq][SPLIT_SLOT_FLOATS]
   uint32_t* split_counters;       // [n_seq * ctrs_per_seq], zero between launches
 };

@@ -106,7 +106,8 @@ int build_plan(const Schedule& S, int layout, Plan* out) {
 
   if (layout == HEATKV_LAYOUT_PAGED) {
     // Pages of 64 rows.  The sink scales of a head share one block of ceil(c_s/64) pages; every
-    // other head-scale owns ceil(t_i/64) pages from its append until its eviction.  Lowest
+    // other head-scale owns ceil(t_i/64) pages from its append until its eviction (a page freed after a
+    // layer is reusable from the next layer's append on).  Lowest
     // free page first, so the highest page ever used equals the peak number of live pages.
     std::priority_queue<int, std::vector<int>, std::greater<int>> free_pages;
     int next_page = 0;
@@ -155,12 +156,6 @@ int build_plan(const Schedule& S, int layout, Plan* out) {
           B.attn_cnt[u] = (int32_t)B.descs.size() - B.attn_begin[u];
         }
         if (k + 1 < K) {
-          for (int h = 0; h < H; ++h) {        // frees first, so the appends can reuse the pages
-            int hd = l * H + h;
-            uint16_t keep = S.keep_mask[S.at(k, l, h)];
-            uint16_t gone = (uint16_t)(stored[hd] & ~keep);
-            if (gone) { release(hd, gone); live_tokens -= tokens_of(gone); stored[hd] &= keep; }
-          }
           for (int h = 0; h < H; ++h) {
             int hd = l * H + h;
             size_t u = S.at(k, l, h);
@@ -180,6 +175,14 @@ int build_plan(const Schedule& S, int layout, Plan* out) {
               live_tokens += S.t[k];
             }
             B.app_cnt[u] = (int32_t)B.descs.size() - B.app_begin[u];
+          }
+          // Pages evicted after this layer are released only now: the new scale never lands on a page the
+          // same step's attention still reads, so the append may run inside the attention launch.
+          for (int h = 0; h < H; ++h) {
+            int hd = l * H + h;
+            uint16_t keep = S.keep_mask[S.at(k, l, h)];
+            uint16_t gone = (uint16_t)(stored[hd] & ~keep);
+            if (gone) { release(hd, gone); live_tokens -= tokens_of(gone); stored[hd] &= keep; }
           }
         }
         out->tokens_post[(size_t)k * L + l] = live_tokens;

@@ -21,6 +21,7 @@ __all__ = [
     "heatkv_create", "heatkv_destroy", "heatkv_calibrate_scores", "heatkv_calibrate_scores_static",
     "heatkv_finalize_scores", "heatkv_build_schedule", "heatkv_schedule_free", "heatkv_schedule_masks", "heatkv_schedule_footprint",
     "heatkv_schedule_plan", "heatkv_seq_open", "heatkv_seq_close", "heatkv_append_compact", "heatkv_scale_attention",
+    "heatkv_attention_append",
     "heatkv_cache_bytes", "heatkv_retained_indices", "heatkv_export_head", "heatkv_allocator_stats",
     "heatkv_launch_count", "heatkv_device_status", "heatkv_strerror", "heatkv_attention_split", "arena_bytes_for",
 ]
@@ -90,7 +91,7 @@ def exported_symbols():
             "heatkv_finalize_scores",
             "heatkv_build_schedule", "heatkv_schedule_free", "heatkv_schedule_masks",
             "heatkv_schedule_footprint", "heatkv_schedule_plan", "heatkv_seq_open", "heatkv_seq_close", "heatkv_append_compact",
-            "heatkv_scale_attention", "heatkv_cache_bytes", "heatkv_retained_indices", "heatkv_export_head",
+            "heatkv_scale_attention", "heatkv_attention_append", "heatkv_cache_bytes", "heatkv_retained_indices", "heatkv_export_head",
             "heatkv_attention_split", "heatkv_allocator_stats", "heatkv_launch_count", "heatkv_device_status",
             "heatkv_strerror"]
 
@@ -122,6 +123,8 @@ _lib.heatkv_seq_close.argtypes = [_P, C.c_int]
 _lib.heatkv_append_compact.argtypes = [_P, C.POINTER(C.c_int), C.c_int, C.c_int, C.c_int, _P, _P, C.POINTER(Strides), _P]
 _lib.heatkv_scale_attention.argtypes = [_P, C.POINTER(C.c_int), C.c_int, C.c_int, C.c_int, _P, _P, _P,
                                         C.POINTER(Strides), _P, _P, _P]
+_lib.heatkv_attention_append.argtypes = [_P, C.POINTER(C.c_int), C.c_int, C.c_int, C.c_int, _P, _P, _P,
+                                         C.POINTER(Strides), _P, _P, _P]
 _lib.heatkv_attention_split.argtypes = [_P, C.POINTER(C.c_int), C.c_int, C.c_int, C.c_int, C.POINTER(C.c_int32),
                                         C.POINTER(C.c_int32)]
 _lib.heatkv_cache_bytes.argtypes = [_P, C.c_int, C.POINTER(C.c_uint64), C.POINTER(C.c_uint64)]
@@ -268,6 +271,14 @@ def heatkv_scale_attention(ctx, seq_ids, layer, step, q, k_new, v_new, strides, 
     st = C.byref(strides) if strides is not None else None
     _check(_lib.heatkv_scale_attention(ctx, ids, n, layer, step, _ptr(q), _ptr(k_new), _ptr(v_new), st,
                                        _ptr(seg_bias), _ptr(out), _stream(stream)), "heatkv_scale_attention")
+
+
+def heatkv_attention_append(ctx, seq_ids, layer, step, q, k_new, v_new, strides, seg_bias, out, stream=None) -> None:
+    """Attention of the layer at the step followed by its cache update, one launch in the paged layout."""
+    ids, n = _ids(seq_ids)
+    st = C.byref(strides) if strides is not None else None
+    _check(_lib.heatkv_attention_append(ctx, ids, n, layer, step, _ptr(q), _ptr(k_new), _ptr(v_new), st,
+                                        _ptr(seg_bias), _ptr(out), _stream(stream)), "heatkv_attention_append")
 
 
 def heatkv_attention_split(ctx, seq_ids, layer, step):

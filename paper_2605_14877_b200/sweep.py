@@ -47,11 +47,15 @@ class Session:
         lo = self.c[step - 1] if step > 0 else 0
         return lo, self.c[step]
 
-    def run_layer_step(self, seq_ids, layer: int, step: int, q, k, v, out, seg_bias=None) -> None:
-        """q, k, v, out: [n_seq, H, n_tokens, d] tensors holding all scales; uses the slice of `step`."""
+    def run_layer_step(self, seq_ids, layer: int, step: int, q, k, v, out, seg_bias=None, fused: bool = False) -> None:
+        """q, k, v, out: [n_seq, H, n_tokens, d] tensors holding all scales; uses the slice of `step`.
+        `fused`: one heatkv_attention_append call instead of attention followed by the cache update."""
         lo, hi = self.step_slices(step)
         qs, ks, vs, os_ = q[:, :, lo:hi], k[:, :, lo:hi], v[:, :, lo:hi], out[:, :, lo:hi]
         st = hk.Strides.of(qs, ks, os_)
+        if fused:
+            hk.heatkv_attention_append(self.ctx, seq_ids, layer, step, qs, ks, vs, st, seg_bias, os_)
+            return
         hk.heatkv_scale_attention(self.ctx, seq_ids, layer, step, qs, ks, vs, st, seg_bias, os_)
         hk.heatkv_append_compact(self.ctx, seq_ids, layer, step, ks, vs, st)
 
@@ -60,13 +64,13 @@ class Session:
 
     def generate(self, seq_ids, qkv_of_layer: Callable[[int], tuple], out_of_layer: Callable[[int], torch.Tensor],
                  bias_of: Optional[Callable[[int, int], Optional[torch.Tensor]]] = None,
-                 after: Optional[Callable[[int, int], None]] = None) -> None:
+                 after: Optional[Callable[[int, int], None]] = None, fused: bool = False) -> None:
         """Whole sweep: steps outer, layers inner.  `after(step, layer)` runs after each layer."""
         for step in range(self.K):
             self.pre_step(seq_ids, step)
             for layer in range(self.L):
                 q, k, v = qkv_of_layer(layer)
                 bias = bias_of(layer, step) if bias_of else None
-                self.run_layer_step(seq_ids, layer, step, q, k, v, out_of_layer(layer), bias)
+                self.run_layer_step(seq_ids, layer, step, q, k, v, out_of_layer(layer), bias, fused)
                 if after:
                     after(step, layer)

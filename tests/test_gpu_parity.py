@@ -60,7 +60,7 @@ def _check_attention(got_bf16, ref_f64, what, stats=None):
 
 
 def _run_full_parity(hk, sh, ref, make_schedule, layout, seed=0, bias=None, kernel=None, n_seq=None,
-                     check_heads=None, check_cache=True):
+                     check_heads=None, check_cache=True, fused=False):
     """Whole generation of one batch; compares every (seq, layer, head, step) unless check_heads
     restricts the oracle work to a list of (seq, layer, head)."""
     n_seq = sh.n_seq if n_seq is None else n_seq
@@ -92,7 +92,7 @@ def _run_full_parity(hk, sh, ref, make_schedule, layout, seed=0, bias=None, kern
                 assert np.array_equal(W.bf16_bits(vo)[: len(idx)], vv), (step, l, h)
 
         ses.generate(ids, lambda l: layers[l], lambda l: outs[l],
-                     (lambda l, k: bias_dev[l, k]) if bias is not None else None, after)
+                     (lambda l, k: bias_dev[l, k]) if bias is not None else None, after, fused)
         torch.cuda.synchronize()
         assert hk.heatkv_device_status(ses.ctx) == 0
         stats = _ErrStats()
@@ -160,6 +160,32 @@ def test_tensor_memory_kernel_full_cache(hk):
     ref = O.heatkv_schedule(scores, 1.0, sh.s, sh.sides)
     _run_full_parity(hk, sh, ref, lambda ses: ses.schedule(scas=scores, b=1.0), hk.LAYOUT_PAGED,
                      kernel=hk.KERNEL_TCGEN05, check_cache=False)
+
+
+@pytest.mark.parametrize("layout", [0, 1], ids=["ragged", "paged"])
+@pytest.mark.parametrize("kernel", [1, 2], ids=["generic", "tcgen05"])
+def test_attention_with_cache_update_in_one_call(hk, layout, kernel):
+    """heatkv_attention_append: in the paged layout the append rides on the attention launch as extra CTAs
+    (both kernels); outputs, retained indices and cache contents after every layer as with separate calls."""
+    sh = W.Shape("mid", L=2, H=4, d=128, sides=W.SIDES_13[:11], n_seq=2, s=3)
+    scores = W.synthetic_scas(sh, 4)
+    ref = O.heatkv_schedule(scores, 0.15, sh.s, sh.sides)
+    bias = W.seg_bias_prior_lognormal(sh, 3)
+    n = _run_full_parity(hk, sh, ref, lambda ses: ses.schedule(scas=scores, b=0.15), layout, bias=bias, kernel=kernel,
+                         fused=True)
+    if layout == 1:
+        assert n == sh.K * sh.L                      # one launch per (step, layer): every update here is small
+
+
+def test_config2_one_call_per_step_sampled_heads(hk):
+    sh = W.CFG2
+    scores = W.synthetic_scas(sh, 0)
+    ref = O.heatkv_schedule(scores, 0.05, sh.s, sh.sides)
+    bias = W.seg_bias_current_scale(sh, 0)
+    heads = [(0, 0, 1), (1, 0, 6), (1, 0, 12)]
+    n = _run_full_parity(hk, sh, ref, lambda ses: ses.schedule(scas=scores, b=0.05), hk.LAYOUT_PAGED, bias=bias,
+                         kernel=hk.KERNEL_AUTO, check_heads=heads, fused=True)
+    assert n == sh.K
 
 
 def test_key_range_splitting_is_used_and_exact(hk):
