@@ -347,8 +347,9 @@ def test_step_order_and_pool_errors(hk):
 
 
 def test_config2_graph_replay_sampled_heads(hk):
-    """Config 2 at full size in the launch configuration the bench times: the 13-step sweep recorded
-    once into a CUDA graph (per-scale contiguous buffers, default strides) and replayed; outputs of
+    """Config 2 at full size in the launch configuration the bench times: the 13-step sweep (one
+    heatkv_attention_append call per scale) recorded once into a CUDA graph (per-scale contiguous buffers,
+    default strides) and replayed; outputs of
     the replay against the oracle on sampled (seq, head) pairs."""
     from paper_2605_14877_b200.sweep import Session
     sh = W.CFG2
@@ -370,9 +371,8 @@ def test_config2_graph_replay_sampled_heads(hk):
             ids = [hk.heatkv_seq_open(ses.ctx, sch) for _ in range(sh.n_seq)]
             for step in range(sh.K):
                 ses.pre_step(ids, step)
-                hk.heatkv_scale_attention(ses.ctx, ids, 0, step, qs[step], ks[step], vs[step], None, bias[0, step],
-                                          outs[step])
-                hk.heatkv_append_compact(ses.ctx, ids, 0, step, ks[step], vs[step], None)
+                hk.heatkv_attention_append(ses.ctx, ids, 0, step, qs[step], ks[step], vs[step], None, bias[0, step],
+                                           outs[step])
             for i in ids:
                 hk.heatkv_seq_close(ses.ctx, i)
 
