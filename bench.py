@@ -441,10 +441,33 @@ def run_model_workload(args, which):
         torch.cuda.synchronize()
         ms = max(e0.elapsed_time(e1), 1e3 * (time.perf_counter() - t0)) / reps
         assert hk.heatkv_device_status(ses.ctx) == 0
+        # the same generation as one CUDA graph (all launches of all layers and scales), replayed
+        graph_ms = None
+        if args.launch == "graph":
+            side = torch.cuda.Stream()
+            side.wait_stream(torch.cuda.current_stream())
+            with torch.cuda.stream(side):
+                generation(False)
+            torch.cuda.current_stream().wait_stream(side)
+            torch.cuda.synchronize()
+            g = torch.cuda.CUDAGraph()
+            with torch.cuda.graph(g):
+                generation(False)
+            g.replay()
+            torch.cuda.synchronize()
+            e0.record(stream)
+            for _ in range(reps):
+                g.replay()
+            e1.record(stream)
+            torch.cuda.synchronize()
+            graph_ms = e0.elapsed_time(e1) / reps
+            assert hk.heatkv_device_status(ses.ctx) == 0
         n_images = sh.n_seq / (2 if which != "serving" else 1)      # cond/uncond pair = one image outside serving
         full_bytes = sh.n_seq * sh.L * sh.H * sh.c[-2] * sh.d * 4
         results.append({"budgets": sorted(set(round(b, 4) for b in budgets)), "ms_per_generation": round(ms, 2),
                         "images_per_s": round(n_images / (ms * 1e-3), 2),
+                        "graph_ms_per_generation": None if graph_ms is None else round(graph_ms, 2),
+                        "graph_images_per_s": None if graph_ms is None else round(n_images / (graph_ms * 1e-3), 2),
                         "cache_GB_end": round(a.used_tokens * sh.d * 4 / 1e9, 3),
                         "cache_GB_uncompressed": round(full_bytes / 1e9, 3),
                         "reserved_GB": round(a.reserved_rows * sh.d * 4 / 1e9, 3),
@@ -453,7 +476,7 @@ def run_model_workload(args, which):
         for sch in schs.values():
             hk.heatkv_schedule_free(sch)
         ses.close()
-    print(json.dumps({"workload": sh.name, "L": sh.L, "H": sh.H, "n_seq": sh.n_seq, "launch": "eager",
+    print(json.dumps({"workload": sh.name, "L": sh.L, "H": sh.H, "n_seq": sh.n_seq, "launch": "calls issued from Python (ms_per_generation) and one CUDA graph replay (graph_*)",
                       "data": "synthetic, one layer's activations reused by all layers", "runs": results}), flush=True)
 
 

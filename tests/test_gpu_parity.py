@@ -188,6 +188,18 @@ def test_config2_one_call_per_step_sampled_heads(hk):
     assert n == sh.K
 
 
+def test_28_head_layer_width(hk):
+    """A layer width that is not a power of two (28 heads of 128, the width the larger model's cache
+    figures imply): heads beyond the 32-lane prefix chunk, odd head counts in the item tables."""
+    sh = W.Shape("w28", L=1, H=28, d=128, sides=W.SIDES_13[:11], n_seq=2, s=3)
+    scores = W.synthetic_scas(sh, 6)
+    ref = O.heatkv_schedule(scores, 0.1, sh.s, sh.sides)
+    bias = W.seg_bias_prior_lognormal(sh, 6)
+    heads = [(0, 0, 0), (1, 0, 13), (0, 0, 27)]
+    _run_full_parity(hk, sh, ref, lambda ses: ses.schedule(scas=scores, b=0.1), hk.LAYOUT_PAGED, bias=bias,
+                     kernel=hk.KERNEL_AUTO, check_heads=heads, fused=True)
+
+
 def test_key_range_splitting_is_used_and_exact(hk):
     """Few heads with long key ranges: the launch cuts them into pieces that meet in the scratch region
     (checked through heatkv_attention_split), and the merged outputs still match the oracle; a context
