@@ -314,7 +314,7 @@ void choose_split(heatkv_ctx* ctx, const int* seq_ids, int n_seq, int step, int 
       const int cand = (max_tiles + div - 1) / div;
       if (cand < 6) break;                                  // pieces about as short as the fixed cost never pay
       const SplitShape sh = split_shape(pe0, step, layer, own_slots, n_qp, cand);
-      if ((uint64_t)sh.slots * n_seq > ctx->split_slots || (uint64_t)sh.ctrs * n_seq > ctx->split_ctrs) continue;
+      if ((uint64_t)sh.slots * n_seq > ctx->split_slots || (uint64_t)sh.ctrs * n_seq * 8 > ctx->split_ctrs) continue;
       const double t = split_makespan(pe0, step, layer, own_slots, n_qp, n_seq, cand, ctx->n_sm);
       if (t < 0.92 * best) { best = t; lmax = cand; }
     }
@@ -333,7 +333,7 @@ void choose_split(heatkv_ctx* ctx, const int* seq_ids, int n_seq, int step, int 
     return m;
   };
   SplitShape m = bounds(lmax);
-  if (lmax > 0 && ((uint64_t)m.slots * n_seq > ctx->split_slots || (uint64_t)m.ctrs * n_seq > ctx->split_ctrs)) {
+  if (lmax > 0 && ((uint64_t)m.slots * n_seq > ctx->split_slots || (uint64_t)m.ctrs * n_seq * 8 > ctx->split_ctrs)) {
     lmax = 0;                                               // another schedule in the batch needs more scratch: whole heads
     m = bounds(0);
   }

@@ -46,7 +46,8 @@ struct AttnParams {
   int16_t table_head[64];
   int16_t table_tiles[64];
   int32_t append_tiles;           // > 0: the launch also stores the step's K/V (paged layout): that many destination
-                                  // half-tile slots per (sequence, head) run as extra CTAs after the attention CTAs
+                                  // half-tile slots per (sequence, head) follow the attention work
+  int32_t attn_items, store_items;  // tensor-memory kernel: attention work items; cache-update items (destination half-tiles)
   float* split_partials;          // [n_seq * slots_per_seq][SPLIT_SLOT_FLOATS]
   uint32_t* split_counters;       // [n_seq * ctrs_per_seq], zero between launches
 };
