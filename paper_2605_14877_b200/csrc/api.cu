@@ -98,6 +98,13 @@ inline bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 
 
 }  // namespace
 
+// How one attention launch cuts its heads: pieces per head in dispatch order; `lmax` > 0 when that is the
+// same as "no run longer than lmax tiles" (the rule a call with several schedules applies to all of them).
+struct SplitChoice {
+  std::vector<int> ns;
+  int lmax = 0;
+};
+
 struct heatkv_ctx {
   heatkv_config cfg;
   int c[HEATKV_MAX_K];
@@ -119,7 +126,7 @@ struct heatkv_ctx {
   uint32_t* split_counters = nullptr;
   uint64_t split_slots = 0, split_ctrs = 0;
   int n_sm = 148;
-  std::map<uint64_t, int> split_choice;     // (plan uid, step, layer, n_seq) -> longest run of tiles per CTA (0: whole heads)
+  std::map<uint64_t, SplitChoice> split_choice;   // (plan uid, step, layer, n_seq) -> pieces per head of the attention launch
 };
 
 namespace {
@@ -237,45 +244,51 @@ int gather_seqs(heatkv_ctx* ctx, const int* seq_ids, int n_seq, int layer, int s
 }
 
 // ---- key-range splitting of the tensor-memory attention kernel -----------------------------------------
-// Items of one sequence under a longest run of `lmax` tiles (0: whole heads): count, partial slots, counters.
+// Items of one sequence: count, partial slots, counters.
 struct SplitShape {
   int items = 0, slots = 0, ctrs = 0;
 };
 
-SplitShape split_shape(const PlanEntry& pe, int step, int layer, int own_slots, int n_qp, int lmax) {
-  const Schedule& s = pe.sched;
-  const PlanHeader& h = pe.plan.header();
-  const int32_t* cnt = pe.plan.blob.data() + h.off_attn_cnt + s.at(step, layer, 0);
-  SplitShape r;
-  for (int hd = 0; hd < s.H; ++hd) {
-    const int tiles = (cnt[hd] + own_slots + 1) / 2;
-    const int ns = lmax > 0 ? (tiles + lmax - 1) / lmax : 1;
-    r.items += n_qp * ns;
-    if (ns > 1) { r.slots += n_qp * ns; r.ctrs += n_qp; }
-  }
-  return r;
-}
-
-// Estimated makespan (in units of one 128-key tile) of the launch when no CTA takes more than `lmax` tiles.
-// Items are handed to the SMs in dispatch order (heads by descending key count, pieces, query tile pairs,
-// sequences interleaved); for very large launches the list-scheduling bound total / SMs + longest is used.
-// The per-CTA constants were fitted to timings of launches with 2 to 32 (sequence, head) units.
-double split_makespan(const PlanEntry& pe, int step, int layer, int own_slots, int n_qp, int n_seq, int lmax, int n_sm) {
-  constexpr double FIXED = 6.0, PUBLISH = 1.5, MERGE_PER_PIECE = 1.5;
+// Key tiles of the heads of (step, layer), in the plan's dispatch order (descending key count).
+std::vector<int> ordered_tiles(const PlanEntry& pe, int step, int layer, int own_slots) {
   const Schedule& s = pe.sched;
   const PlanHeader& h = pe.plan.header();
   const int32_t* blob = pe.plan.blob.data();
   const int32_t* cnt = blob + h.off_attn_cnt + s.at(step, layer, 0);
   const int32_t* order = blob + h.off_order + s.at(step, layer, 0);
+  std::vector<int> t(s.H);
+  for (int i = 0; i < s.H; ++i) t[i] = (cnt[order[i]] + own_slots + 1) / 2;
+  return t;
+}
+
+// Pieces of a head under a longest run of `lmax` tiles (0: the whole head).
+inline int pieces_for(int tiles, int lmax) { return lmax > 0 ? (tiles + lmax - 1) / lmax : 1; }
+// Every piece of an equal cut must hold at least one tile.
+inline bool cut_ok(int tiles, int ns) { return ns >= 1 && (ns - 1) * ((tiles + ns - 1) / ns) < tiles; }
+
+SplitShape shape_of(const std::vector<int>& tiles, const std::vector<int>& ns, int n_qp) {
+  SplitShape r;
+  for (size_t i = 0; i < tiles.size(); ++i) {
+    r.items += n_qp * ns[i];
+    if (ns[i] > 1) { r.slots += n_qp * ns[i]; r.ctrs += n_qp; }
+  }
+  return r;
+}
+
+// Estimated makespan (in units of one 128-key tile) of the launch.  Items are taken by the resident CTAs in
+// dispatch order (heads by descending key count, pieces, query tile pairs, sequences interleaved); for very
+// large launches the list-scheduling bound total / SMs + longest is used.  The per-item constants were fitted
+// to clock stamps of the kernel: an item costs its tiles plus the result's way out and the next item's start;
+// a piece writes fp32 partials instead, and the piece that arrives last reads the others.
+double makespan_of(const std::vector<int>& tiles, const std::vector<int>& ns, int n_qp, int n_seq, int n_sm) {
+  constexpr double FIXED = 2.0, PUBLISH = 1.0, MERGE_PER_PIECE = 1.5;
   std::vector<double> costs;
   double total = 0.0, longest = 0.0;
-  for (int i = 0; i < s.H; ++i) {
-    const int tiles = (cnt[order[i]] + own_slots + 1) / 2;
-    const int ns = lmax > 0 ? (tiles + lmax - 1) / lmax : 1;
-    const int piece = (tiles + ns - 1) / ns;
-    for (int pc = 0; pc < ns; ++pc) {
-      const int len = std::min(tiles, (pc + 1) * piece) - pc * piece;
-      const double c = len + FIXED + (ns > 1 ? PUBLISH + MERGE_PER_PIECE * (ns - 1) / ns : 0.0);
+  for (size_t i = 0; i < tiles.size(); ++i) {
+    const int piece = (tiles[i] + ns[i] - 1) / ns[i];
+    for (int pc = 0; pc < ns[i]; ++pc) {
+      const int len = std::min(tiles[i], (pc + 1) * piece) - pc * piece;
+      const double c = len + FIXED + (ns[i] > 1 ? PUBLISH + MERGE_PER_PIECE * (ns[i] - 1) / ns[i] : 0.0);
       for (int q = 0; q < n_qp; ++q) costs.push_back(c);
       total += c * n_qp;
       longest = std::max(longest, c);
@@ -294,66 +307,97 @@ double split_makespan(const PlanEntry& pe, int step, int layer, int own_slots, i
   return *std::max_element(sm.begin(), sm.end());
 }
 
-// Fills the splitting fields of the launch parameters.  The choice is cached per (schedule, step, layer,
-// batch size); sequences of other schedules in the same call only raise the per-sequence bounds.
+// Fills the splitting fields of the launch parameters.  When the whole call follows one schedule the choice
+// is a piece count per head: long heads are cut to a common longest run, and the heads dispatched last may be
+// cut further so that the last round of items fills the SMs.  It is cached per (schedule, step, layer, batch
+// size).  Calls that mix schedules use one longest run for all of them.
 void choose_split(heatkv_ctx* ctx, const int* seq_ids, int n_seq, int step, int layer, AttnParams* p) {
+  constexpr int MIN_PIECE = 6;                              // pieces about as short as the fixed cost never pay
   const int n_qp = (p->t_q + 255) / 256, own_slots = (p->n_own + HEATKV_PAGE_TOKENS - 1) / HEATKV_PAGE_TOKENS;
   const PlanEntry& pe0 = *ctx->plans[ctx->seqs[seq_ids[0]].plan];
-  const uint64_t key = (pe0.uid << 24) ^ ((uint64_t)step << 20) ^ ((uint64_t)layer << 8) ^ (uint64_t)n_seq;
-  int lmax = 0;
+  bool one_plan = pe0.sched.H <= 64;
+  for (int i = 1; i < n_seq && one_plan; ++i) one_plan = ctx->seqs[seq_ids[i]].plan == ctx->seqs[seq_ids[0]].plan;
+  const std::vector<int> tiles = ordered_tiles(pe0, step, layer, own_slots);
+  const int H = (int)tiles.size();
+  for (int t : tiles) one_plan = one_plan && t <= 32767;
+  const uint64_t key = (pe0.uid << 24) ^ ((uint64_t)step << 20) ^ ((uint64_t)layer << 8) ^ (uint64_t)n_seq ^
+                       (one_plan ? 0ull : 1ull << 63);
+  auto fits = [&](const SplitShape& sh) {
+    return (uint64_t)sh.slots * n_seq <= ctx->split_slots && (uint64_t)sh.ctrs * n_seq * 8 <= ctx->split_ctrs;
+  };
   auto it = ctx->split_choice.find(key);
-  if (it != ctx->split_choice.end()) {
-    lmax = it->second;
-  } else {
-    const Schedule& s = pe0.sched;
-    const int32_t* cnt = pe0.plan.blob.data() + pe0.plan.header().off_attn_cnt + s.at(step, layer, 0);
-    int max_tiles = 1;
-    for (int hd = 0; hd < s.H; ++hd) max_tiles = std::max(max_tiles, (cnt[hd] + own_slots + 1) / 2);
-    double best = split_makespan(pe0, step, layer, own_slots, n_qp, n_seq, 0, ctx->n_sm);
+  if (it == ctx->split_choice.end()) {
+    SplitChoice best;
+    best.ns.assign(H, 1);
+    double best_t = makespan_of(tiles, best.ns, n_qp, n_seq, ctx->n_sm);
+    const int max_tiles = *std::max_element(tiles.begin(), tiles.end());
+    std::vector<int> lmaxes = {0};
     for (int div : {2, 3, 4, 6, 8, 12, 16}) {
       const int cand = (max_tiles + div - 1) / div;
-      if (cand < 6) break;                                  // pieces about as short as the fixed cost never pay
-      const SplitShape sh = split_shape(pe0, step, layer, own_slots, n_qp, cand);
-      if ((uint64_t)sh.slots * n_seq > ctx->split_slots || (uint64_t)sh.ctrs * n_seq * 8 > ctx->split_ctrs) continue;
-      const double t = split_makespan(pe0, step, layer, own_slots, n_qp, n_seq, cand, ctx->n_sm);
-      if (t < 0.92 * best) { best = t; lmax = cand; }
+      if (cand < MIN_PIECE) break;
+      lmaxes.push_back(cand);
     }
-    ctx->split_choice[key] = lmax;
+    for (int lmax : lmaxes) {
+      std::vector<int> base(H);
+      for (int i = 0; i < H; ++i) base[i] = pieces_for(tiles[i], lmax);
+      // heads dispatched last (the shortest) cut into `extra` times as many pieces; only with a per-head table
+      for (int extra = 1; extra <= (one_plan ? 3 : 1); ++extra)
+        for (int tail = (extra == 1 ? 0 : 1); tail <= (extra == 1 ? 0 : H); ++tail) {
+          std::vector<int> ns = base;
+          bool ok = true;
+          for (int i = H - tail; i < H; ++i) {
+            ns[i] = base[i] * extra;
+            ok = ok && cut_ok(tiles[i], ns[i]) && (tiles[i] + ns[i] - 1) / ns[i] >= MIN_PIECE;
+          }
+          for (int i = 0; i < H; ++i) ok = ok && cut_ok(tiles[i], ns[i]);
+          if (!ok || (lmax == 0 && tail == 0)) continue;
+          if (!fits(shape_of(tiles, ns, n_qp))) continue;
+          const double t = makespan_of(tiles, ns, n_qp, n_seq, ctx->n_sm);
+          if (t < 0.95 * best_t) { best_t = t; best.ns = ns; best.lmax = tail == 0 ? lmax : -1; }
+        }
+    }
+    it = ctx->split_choice.emplace(key, std::move(best)).first;
   }
-  auto bounds = [&](int lm) {
-    SplitShape m;
-    int last_plan = -1;
-    for (int i = 0; i < n_seq; ++i) {
-      const int pi = ctx->seqs[seq_ids[i]].plan;
-      if (pi == last_plan) continue;
-      last_plan = pi;
-      const SplitShape sh = split_shape(*ctx->plans[pi], step, layer, own_slots, n_qp, lm);
-      m.items = std::max(m.items, sh.items); m.slots = std::max(m.slots, sh.slots); m.ctrs = std::max(m.ctrs, sh.ctrs);
+  const SplitChoice& ch = it->second;
+  SplitShape m = shape_of(tiles, ch.ns, n_qp);
+  int lmax = ch.lmax > 0 ? ch.lmax : 0;
+  if (!one_plan) {
+    // other schedules in the batch follow the same longest run; the per-sequence bounds cover all of them
+    auto bounds = [&](int lm) {
+      SplitShape b;
+      int last_plan = -1;
+      for (int i = 0; i < n_seq; ++i) {
+        const int pi = ctx->seqs[seq_ids[i]].plan;
+        if (pi == last_plan) continue;
+        last_plan = pi;
+        const std::vector<int> t = ordered_tiles(*ctx->plans[pi], step, layer, own_slots);
+        std::vector<int> ns(t.size());
+        for (size_t k = 0; k < t.size(); ++k) ns[k] = pieces_for(t[k], lm);
+        const SplitShape sh = shape_of(t, ns, n_qp);
+        b.items = std::max(b.items, sh.items); b.slots = std::max(b.slots, sh.slots); b.ctrs = std::max(b.ctrs, sh.ctrs);
+      }
+      return b;
+    };
+    m = bounds(lmax);
+    if (lmax > 0 && !fits(m)) {
+      lmax = 0;                                             // another schedule in the batch needs more scratch: whole heads
+      m = bounds(0);
     }
-    return m;
-  };
-  SplitShape m = bounds(lmax);
-  if (lmax > 0 && ((uint64_t)m.slots * n_seq > ctx->split_slots || (uint64_t)m.ctrs * n_seq * 8 > ctx->split_ctrs)) {
-    lmax = 0;                                               // another schedule in the batch needs more scratch: whole heads
-    m = bounds(0);
   }
   // one plan for the whole call (the usual case): its heads, by descending key count, travel in the parameters
   p->table_heads = 0;
-  bool one_plan = pe0.sched.H <= 64;
-  for (int i = 1; i < n_seq && one_plan; ++i) one_plan = ctx->seqs[seq_ids[i]].plan == ctx->seqs[seq_ids[0]].plan;
+  p->longest_piece = 0;
   if (one_plan) {
-    const Schedule& s = pe0.sched;
-    const int32_t* blob = pe0.plan.blob.data();
-    const int32_t* cnt = blob + pe0.plan.header().off_attn_cnt + s.at(step, layer, 0);
-    const int32_t* order = blob + pe0.plan.header().off_order + s.at(step, layer, 0);
-    bool fits = true;
-    for (int i = 0; i < s.H; ++i) {
-      const int tiles = (cnt[order[i]] + own_slots + 1) / 2;
-      fits = fits && tiles <= 32767;
+    const int32_t* order = pe0.plan.blob.data() + pe0.plan.header().off_order + pe0.sched.at(step, layer, 0);
+    for (int i = 0; i < H; ++i) {
       p->table_head[i] = (int16_t)order[i];
-      p->table_tiles[i] = (int16_t)tiles;
+      p->table_tiles[i] = (int16_t)tiles[i];
+      p->table_split[i] = (int16_t)ch.ns[i];
+      if (ch.ns[i] > 1) p->longest_piece = std::max(p->longest_piece, (tiles[i] + ch.ns[i] - 1) / ch.ns[i]);
     }
-    if (fits) p->table_heads = s.H;
+    p->table_heads = H;
+  } else {
+    p->longest_piece = lmax;
   }
   p->n_seq = n_seq;
   p->split_tiles = lmax;
@@ -668,7 +712,7 @@ int heatkv_attention_split(heatkv_ctx* ctx, const int* seq_ids, int n_seq, int l
   } catch (const std::bad_alloc&) {
     return HEATKV_ERR_HOST_MEMORY;
   }
-  if (split_tiles) *split_tiles = p.split_tiles;
+  if (split_tiles) *split_tiles = p.longest_piece;
   if (items) *items = p.items_per_seq * n_seq;
   return HEATKV_OK;
 }

@@ -226,8 +226,9 @@ attn_tc_kernel(const __grid_constant__ AttnParams p, const __grid_constant__ Map
         break;
       }
       // Attention items: sequences interleaved; the items of one sequence run over its heads by descending
-      // key count (the plan's order); a head whose key range exceeds split_tiles tiles is cut into equal
-      // pieces, and every (piece, query tile pair) is one item, pieces outermost.  A prefix sum over the
+      // key count (the plan's order); a head may be cut into equal pieces of its key range (the count comes
+      // from the host's table, else from the launch's longest run), and every (piece, query tile pair) is
+      // one item, pieces outermost.  A prefix sum over the
       // heads finds the item.
       const int seq = idx % p.n_seq;
       const int item = idx / p.n_seq;
@@ -242,11 +243,12 @@ attn_tc_kernel(const __grid_constant__ AttnParams p, const __grid_constant__ Map
           if (p.table_heads > 0) {                            // the host put the per-head table into the launch parameters
             h = p.table_head[i];
             tiles = p.table_tiles[i];
+            ns = p.table_split[i];
           } else {
             h = pv.order()[u + i];
             tiles = (pv.attn_cnt()[u + h] + own_slots + 1) >> 1;
+            ns = p.split_tiles > 0 ? (tiles + p.split_tiles - 1) / p.split_tiles : 1;
           }
-          ns = p.split_tiles > 0 ? (tiles + p.split_tiles - 1) / p.split_tiles : 1;
           cnt = n_qp * ns;
         }
         const int scnt = ns > 1 ? cnt : 0, ccnt = ns > 1 ? n_qp : 0;
@@ -660,16 +662,23 @@ attn_tc_kernel(const __grid_constant__ AttnParams p, const __grid_constant__ Map
           if (ok && im.n_split == 1) {
             tc_fence_after();
             const float inv = 1.f / l_sum;
-#pragma unroll 1
-            for (int c = 0; c < 4; ++c) {
-              uint32_t r[32];
-              tmem_ld32(t_o + c * 32, r);
-              tmem_wait_ld();
+            // the whole row of O in one go, so the four groups' conversions and stores overlap
+            uint32_t o0[32], o1[32], o2[32], o3[32];
+            tmem_ld32(t_o, o0);
+            tmem_ld32(t_o + 32, o1);
+            tmem_ld32(t_o + 64, o2);
+            tmem_ld32(t_o + 96, o3);
+            tmem_wait_ld();
+            auto out_group = [&](const uint32_t (&r)[32], int c) {
               float acc[32];
 #pragma unroll
               for (int i = 0; i < 32; ++i) acc[i] = __uint_as_float(r[i]);
               store_rows(acc, inv, c);
-            }
+            };
+            out_group(o0, 0);
+            out_group(o1, 1);
+            out_group(o2, 2);
+            out_group(o3, 3);
           } else if (ok) {
             // A piece of a split head: publish the unnormalised O of this row with its reference and row
             // sum; the warp that arrives last at the counter of these 32 rows merges

@@ -41,10 +41,12 @@ struct AttnParams {
   int32_t items_per_seq;          // work items (head, piece, query tile pair) of one sequence, an upper bound
   int32_t slots_per_seq;          // partial-result slots reserved per sequence
   int32_t ctrs_per_seq;           // arrival counters reserved per sequence
-  int32_t table_heads;            // > 0: every sequence of the call follows one plan and the two tables below hold,
-                                  // for its heads by descending key count, the head index and its number of key tiles
+  int32_t table_heads;            // > 0: every sequence of the call follows one plan and the tables below hold, for
+                                  // its heads by descending key count, the head index, its key tiles and its pieces
   int16_t table_head[64];
   int16_t table_tiles[64];
+  int16_t table_split[64];        // pieces the head's key range is cut into (1: whole head)
+  int32_t longest_piece;          // host report: longest piece among the heads that are cut (0: none is)
   int32_t append_tiles;           // > 0: the launch also stores the step's K/V (paged layout): that many destination
                                   // half-tile slots per (sequence, head) follow the attention work
   int32_t attn_items, store_items;  // tensor-memory kernel: attention work items; cache-update items (destination half-tiles)
