@@ -41,6 +41,8 @@ namespace {
 
 constexpr uint64_t META_ALIGN = 256;
 constexpr uint64_t STATUS_BYTES = 256;
+// largest cache update (bytes read + written) that rides on the attention launch, per kernel
+constexpr uint64_t FUSE_LIMIT_TC_BYTES = 1ull << 30, FUSE_LIMIT_GENERIC_BYTES = 8ull << 20;
 
 // first-fit allocator over [0, size) in abstract units
 struct RangeAlloc {
@@ -645,24 +647,25 @@ static int attention_impl(heatkv_ctx* ctx, const int* seq_ids, int n_seq, int la
   p.step = step;
   p.layer = layer;
   const bool stores = step + 1 < ctx->cfg.K;                  // the last scale is never cached
+  const int choice = ctx->cfg.kernel;
+  bool use_tc = choice != HEATKV_KERNEL_GENERIC && tc_supported(ctx->tc, p, ctx->cfg.d, n_seq, false);
+  if (choice == HEATKV_KERNEL_AUTO && p.t_q < 256) use_tc = false;
+  if (choice == HEATKV_KERNEL_TCGEN05 && !use_tc) return HEATKV_ERR_INVALID_ARG;   // never a silent substitute
   bool fuse = with_update && stores && ctx->cfg.layout == HEATKV_LAYOUT_PAGED;
   if (fuse) {
-    // The append rides on the attention launch only while it is small (a launch-bound copy): its CTAs share
-    // the attention kernel's one-CTA-per-SM footprint, so a bandwidth-sized append keeps its own kernel.
-    constexpr uint64_t FUSE_LIMIT_BYTES = 8u << 20;
+    // The tensor-memory kernel copies the new rows with two spare warps per SM beside the attention work, so
+    // the update rides along whatever its size.  The generic kernel carries it as extra CTAs of its own
+    // footprint, which only pays while the update is a launch-bound copy; a larger one keeps its own kernel.
+    const uint64_t limit = use_tc ? FUSE_LIMIT_TC_BYTES : FUSE_LIMIT_GENERIC_BYTES;
     uint64_t storing = 0;
     for (int i = 0; i < n_seq; ++i) {
       const PlanEntry& pe = *ctx->plans[ctx->seqs[seq_ids[i]].plan];
       const int32_t* cnt = pe.plan.blob.data() + pe.plan.header().off_app_cnt + pe.sched.at(step, layer, 0);
       for (int hd = 0; hd < pe.sched.H; ++hd) storing += cnt[hd] > 0;
     }
-    fuse = storing * (uint64_t)ctx->cfg.t[step] * ctx->cfg.d * 8 <= FUSE_LIMIT_BYTES;
+    fuse = storing * (uint64_t)ctx->cfg.t[step] * ctx->cfg.d * 8 <= limit;
   }
   if (fuse) p.append_tiles = (ctx->cfg.t[step] + HEATKV_PAGE_TOKENS - 1) / HEATKV_PAGE_TOKENS + 1;
-  const int choice = ctx->cfg.kernel;
-  bool use_tc = choice != HEATKV_KERNEL_GENERIC && tc_supported(ctx->tc, p, ctx->cfg.d, n_seq, false);
-  if (choice == HEATKV_KERNEL_AUTO && p.t_q < 256) use_tc = false;
-  if (choice == HEATKV_KERNEL_TCGEN05 && !use_tc) return HEATKV_ERR_INVALID_ARG;   // never a silent substitute
   cudaError_t e;
   if (use_tc) {
     int n = 0;

@@ -409,8 +409,8 @@ attn_tc_kernel(const __grid_constant__ AttnParams p, const __grid_constant__ Map
           __syncwarp();
         }
         // Waits for K and V sit where the tensor pipe still has queued work: the next tile's V at the end
-        // of an iteration, the next tile's K between PV_A and S_A.  The hand-over of P is then the only
-        // wait between the last S product of one tile and the first PV product of the next.
+        // of an iteration, the next tile's K between the two halves of PV_A.  The hand-over of P is then
+        // the only wait between the last S product of one tile and the first PV product of the next.
         if (ok) ok = warp_wait(bar(V_FULL + st0), par0, abort_flag, p.status);
         for (int j = 0; j < n_tiles && ok; ++j) {
           const uint32_t st = (g + j) % KV_STAGES, stn = (g + j + 1) % KV_STAGES;
@@ -425,6 +425,9 @@ attn_tc_kernel(const __grid_constant__ AttnParams p, const __grid_constant__ Map
             tc_fence_after();
             if (leader) issue_pv(x, st, 0, j == 0);
             __syncwarp();
+            // the next tile's keys are waited for here, off the path between the last half of P and the next S
+            if (more && x == 0) ok = warp_wait(bar(K_FULL + stn), parn, abort_flag, p.status);
+            if (!ok) continue;
             ok = warp_wait(bar(P_FULL + 2 * x + 1), ph, abort_flag, p.status);
             if (!ok) continue;
             tc_fence_after();
@@ -434,8 +437,6 @@ attn_tc_kernel(const __grid_constant__ AttnParams p, const __grid_constant__ Map
             }
             __syncwarp();
             if (more) {
-              if (x == 0) ok = warp_wait(bar(K_FULL + stn), parn, abort_flag, p.status);
-              if (!ok) continue;
               if (leader) {
                 issue_s(x, stn);
                 tc_commit(bar(S_FULL + x));
