@@ -40,7 +40,7 @@ METRIC = "images_per_sec_scale_step_attention_2b_single_layer_20x"
 UNIT = "images/s"
 # dram__bytes_read.sum + dram__bytes_write.sum of the dominant kernel's launches of one sweep, from the ncu
 # capture summarised under profiles/; None once the kernel changed after the capture
-TRAFFIC_BYTES_PER_SWEEP = 306.3e6
+TRAFFIC_BYTES_PER_SWEEP = 318.9e6
 
 
 def peaks():
@@ -657,6 +657,11 @@ def main():
     clocks = sampler.stop()
     per_step_ms = np.array([[ke[kk][0].elapsed_time(ke[kk][1]) for kk in range(shape.K)] for ke in kern_events])
     assert hk.heatkv_device_status(ses.ctx) == 0
+    # how the tensor-memory launches cut their work (host-side report of the library's choice)
+    ids_ = [hk.heatkv_seq_open(ses.ctx, sch) for _ in range(n_seq)]
+    cuts = [hk.heatkv_attention_split(ses.ctx, ids_, 0, kk) for kk in range(shape.K)]
+    for i in ids_:
+        hk.heatkv_seq_close(ses.ctx, i)
 
     # ---- end to end: the same sweep from pinned host buffers, copies inside the timed region
     h2d = 3 * sum(x.numel() for x in qs_) * 2
@@ -717,6 +722,8 @@ def main():
                    "n_k": [int(x) for x in nk], "replicas": world},
         "effective_kv_tb_per_s": uncompressed_kv_bytes / (float(attn_ms.sum()) * 1e-3) / 1e12,
         "attention_ms_per_scale": [round(float(x), 5) for x in attn_ms],
+        "work_items_per_scale": [int(c[1]) for c in cuts],
+        "longest_piece_tiles_per_scale": [int(c[0]) for c in cuts],
         "attention_tflops_per_scale": [round(flops[kk] / (float(attn_ms[kk]) * 1e-3) / 1e12, 1) for kk in range(shape.K)],
         "attention_tflops_all_scales": sum(flops) / (float(attn_ms.sum()) * 1e-3) / 1e12,
         "images_per_s_32_layers_extrapolated": value / 32.0,

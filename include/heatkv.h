@@ -222,21 +222,23 @@ int heatkv_scale_attention(heatkv_ctx* ctx, const int* seq_ids /*HOST*/, int n_s
 
 /* heatkv_scale_attention followed by heatkv_append_compact(k_new != NULL) for the same (layer, step), as one
  * call: the order a model issues them in (Sec. 3.3: evictions "immediately after their layer has executed").
- * In the paged layout both run in ONE kernel launch while the update is small (up to 8 MiB of K/V, a
- * launch-bound copy): its copies are extra CTAs of the attention launch (the plan releases the pages of G_step \ A_step only after the layer's append, so the new
- * scale never lands on a page this step's attention still reads).  Larger updates keep their own
- * bandwidth-bound kernel, and in the ragged layout the in-place compaction must follow the attention, so
+ * In the paged layout both run in ONE kernel launch (the plan releases the pages of G_step \ A_step only
+ * after the layer's append, so the new scale never lands on a page this step's attention still reads): on
+ * the tensor-memory kernel two spare warps per SM copy the new rows beside the attention work, whatever the
+ * update's size; on the generic kernel the copies are extra CTAs of the attention launch while the update
+ * is small (up to 8 MiB of K/V, a launch-bound copy), and a larger update keeps its own bandwidth-bound
+ * kernel.  In the ragged layout the in-place compaction must follow the attention, so
  * there the separate kernels run.  Arguments as in heatkv_scale_attention. */
 int heatkv_attention_append(heatkv_ctx* ctx, const int* seq_ids /*HOST*/, int n_seq, int layer, int step,
                             const void* q, const void* k_new, const void* v_new, const heatkv_strides* st,
                             const float* seg_bias, void* out, void* stream);
 
 /* How the tensor-memory attention kernel would cut the work of heatkv_scale_attention(seq_ids, layer,
- * step): *split_tiles = longest run of 128-key tiles one CTA takes (0: every CTA takes a whole head's key
- * range), *items = CTAs of the launch.  A head with more tiles than split_tiles is cut into equal pieces
- * whose partial results meet in the arena's scratch region; the piece that arrives last merges them.  The
- * choice minimises an estimate of the launch's makespan over the SMs and is cached per (schedule, step,
- * layer, batch size).  Host only. */
+ * step): *split_tiles = longest piece, in 128-key tiles, among the heads whose key range is cut (0: every
+ * work item takes a whole head's key range), *items = work items of the launch (an upper bound when the
+ * call mixes schedules).  A cut head's pieces leave partial results in the arena's scratch region, where
+ * the last to arrive merges them.  The choice (a piece count per head) minimises an estimate of the launch's
+ * makespan over the SMs and is cached per (schedule, step, layer, batch size).  Host only. */
 int heatkv_attention_split(heatkv_ctx* ctx, const int* seq_ids /*HOST*/, int n_seq, int layer, int step,
                            int32_t* split_tiles, int32_t* items);
 

@@ -1,6 +1,7 @@
 // Append of one destination half-tile (up to 64 rows) of a head's new K and V into the rows the plan
 // assigns (Sec. 3.3: the scale is stored unless (k, l, h) is in G_k).  Shared by the stand-alone append
-// kernel and by the attention kernels, whose launches can carry the append as extra CTAs.
+// kernel and by the attention kernels, whose launches can carry the append (extra CTAs of the generic
+// kernel, spare warps of the tensor-memory kernel).
 #pragma once
 #include "device_common.cuh"
 

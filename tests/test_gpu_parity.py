@@ -165,7 +165,7 @@ def test_tensor_memory_kernel_full_cache(hk):
 @pytest.mark.parametrize("layout", [0, 1], ids=["ragged", "paged"])
 @pytest.mark.parametrize("kernel", [1, 2], ids=["generic", "tcgen05"])
 def test_attention_with_cache_update_in_one_call(hk, layout, kernel):
-    """heatkv_attention_append: in the paged layout the append rides on the attention launch as extra CTAs
+    """heatkv_attention_append: in the paged layout the append rides on the attention launch (extra CTAs or spare warps)
     (both kernels); outputs, retained indices and cache contents after every layer as with separate calls."""
     sh = W.Shape("mid", L=2, H=4, d=128, sides=W.SIDES_13[:11], n_seq=2, s=3)
     scores = W.synthetic_scas(sh, 4)
