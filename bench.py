@@ -673,18 +673,36 @@ def main():
         hout = [torch.empty_like(x).pin_memory() for x in hq]
         dq, dk, dv, do = ([torch.empty_like(x) for x in xs] for xs in (qs_, ks_, vs_, os_))
 
+        # Three streams, as a caller that feeds the library from the host would do: uploads of the later
+        # scales run while the earlier ones compute, and each scale's result goes back as soon as it is done.
+        s_in, s_out = torch.cuda.Stream(), torch.cuda.Stream()
+
         def sweep_e2e():
             ids = [hk.heatkv_seq_open(ses.ctx, sch) for _ in range(n_seq)]
+            s_in.wait_stream(stream)                 # the previous sweep has read its inputs
+            ev_in = []
+            with torch.cuda.stream(s_in):
+                for step in range(shape.K):
+                    for src, dst in ((hq, dq), (hkk, dk), (hv, dv)):
+                        dst[step].copy_(src[step], non_blocking=True)
+                    ev = torch.cuda.Event()
+                    ev.record(s_in)
+                    ev_in.append(ev)
+            stream.wait_stream(s_out)                # the previous sweep's results have left the device
             for step in range(shape.K):
-                for src, dst in ((hq, dq), (hkk, dk), (hv, dv)):
-                    dst[step].copy_(src[step], non_blocking=True)
+                stream.wait_event(ev_in[step])
                 ses.pre_step(ids, step)
                 if args.calls == "fused":
                     hk.heatkv_attention_append(ses.ctx, ids, 0, step, dq[step], dk[step], dv[step], None, bias[0, step], do[step])
                 else:
                     hk.heatkv_scale_attention(ses.ctx, ids, 0, step, dq[step], dk[step], dv[step], None, bias[0, step], do[step])
                     hk.heatkv_append_compact(ses.ctx, ids, 0, step, dk[step], dv[step], None)
-                hout[step].copy_(do[step], non_blocking=True)
+                ev = torch.cuda.Event()
+                ev.record(stream)
+                with torch.cuda.stream(s_out):
+                    s_out.wait_event(ev)
+                    hout[step].copy_(do[step], non_blocking=True)
+            stream.wait_stream(s_out)                # the sweep ends when its last result is on the host
             for i in ids:
                 hk.heatkv_seq_close(ses.ctx, i)
 
