@@ -200,6 +200,18 @@ def test_28_head_layer_width(hk):
                      kernel=hk.KERNEL_AUTO, check_heads=heads, fused=True)
 
 
+def test_40_head_layer_width(hk):
+    """More heads than one 32-lane chunk of the work-item prefix sum in the tensor-memory kernel: items of
+    heads 32..39 are found in the second chunk (sampled heads from both chunks, fused cache update)."""
+    sh = W.Shape("w40", L=1, H=40, d=128, sides=W.SIDES_13[:10], n_seq=2, s=3)
+    scores = W.synthetic_scas(sh, 8)
+    ref = O.heatkv_schedule(scores, 0.2, sh.s, sh.sides)
+    bias = W.seg_bias_prior_lognormal(sh, 8)
+    heads = [(0, 0, 0), (1, 0, 31), (0, 0, 32), (1, 0, 39), (0, 0, 17)]
+    _run_full_parity(hk, sh, ref, lambda ses: ses.schedule(scas=scores, b=0.2), hk.LAYOUT_PAGED, bias=bias,
+                     kernel=hk.KERNEL_AUTO, check_heads=heads, fused=True)
+
+
 def test_key_range_splitting_is_used_and_exact(hk):
     """Few heads with long key ranges: the launch cuts them into pieces that meet in the scratch region
     (checked through heatkv_attention_split), and the merged outputs still match the oracle; a context
