@@ -309,6 +309,27 @@ double makespan_of(const std::vector<int>& tiles, const std::vector<int>& ns, in
   return *std::max_element(sm.begin(), sm.end());
 }
 
+// Head table of a call whose sequences all follow one schedule (generic kernel): heads in dispatch order with
+// the place of their descriptors, so the kernel starts without walking the plan.
+void fill_head_table(heatkv_ctx* ctx, const int* seq_ids, int n_seq, int step, int layer, AttnParams* p) {
+  p->table_heads = 0;
+  const PlanEntry& pe0 = *ctx->plans[ctx->seqs[seq_ids[0]].plan];
+  if (pe0.sched.H > 64) return;
+  for (int i = 1; i < n_seq; ++i)
+    if (ctx->seqs[seq_ids[i]].plan != ctx->seqs[seq_ids[0]].plan) return;
+  const PlanHeader& hdr = pe0.plan.header();
+  const int32_t* blob = pe0.plan.blob.data();
+  const int at = pe0.sched.at(step, layer, 0);
+  const int32_t *order = blob + hdr.off_order + at, *cnt = blob + hdr.off_attn_cnt + at, *begin = blob + hdr.off_attn_begin + at;
+  for (int i = 0; i < pe0.sched.H; ++i) {
+    if (cnt[order[i]] > 32767) return;
+    p->table_head[i] = (int16_t)order[i];
+    p->table_ndesc[i] = (int16_t)cnt[order[i]];
+    p->table_desc_begin[i] = hdr.off_desc + 2 * begin[order[i]];
+  }
+  p->table_heads = pe0.sched.H;
+}
+
 // Fills the splitting fields of the launch parameters.  When the whole call follows one schedule the choice
 // is a piece count per head: long heads are cut to a common longest run, and the heads dispatched last may be
 // cut further so that the last round of items fills the SMs.  It is cached per (schedule, step, layer, batch
@@ -677,6 +698,7 @@ static int attention_impl(heatkv_ctx* ctx, const int* seq_ids, int n_seq, int la
     e = launch_attn_tc(ctx->tc, p, ctx->cfg.d, n_seq, false, stream, &n);
     ctx->launches += n;
   } else {
+    fill_head_table(ctx, seq_ids, n_seq, step, layer, &p);
     e = launch_attn_generic(p, ctx->cfg.d, n_seq, false, stream);
     ctx->launches += 1;
   }

@@ -14,16 +14,18 @@ namespace heatkv {
 constexpr int GM = 64;    // queries per CTA
 constexpr int GN = 64;    // keys per half-tile
 constexpr int GTHREADS = 128;
+constexpr int GSTAGES = 2;   // key/value half-tiles in flight or in use per CTA (3 measured no faster: the small steps are bound by the warp-level MMA rate)
 
 template <int D>
 struct GenericSmem {
   static constexpr int TILE_BYTES = GN * D * 2;
-  // q | k[2] | v[2] | seg_sum[GM][16] | seg_ref[GM][16]
+  // q | k[GSTAGES] | v[GSTAGES] | seg_sum[GM][16] | seg_ref[GM][16]
   static constexpr int Q_OFF = 0;
   static constexpr int K_OFF = GM * D * 2;
-  static constexpr int V_OFF = K_OFF + 2 * TILE_BYTES;
-  static constexpr int SEG_OFF = V_OFF + 2 * TILE_BYTES;
+  static constexpr int V_OFF = K_OFF + GSTAGES * TILE_BYTES;
+  static constexpr int SEG_OFF = V_OFF + GSTAGES * TILE_BYTES;
   static constexpr int BYTES = SEG_OFF + 2 * GM * HEATKV_MAX_K * 4;
+  static constexpr int ATTN_BYTES = SEG_OFF;             // without the calibration sums: two CTAs of head_dim 128 fit an SM
 };
 
 // byte offset of 16-byte chunk `ch` of row `r` in a [rows][D] bf16 tile (XOR swizzle)
@@ -80,11 +82,19 @@ __global__ void __launch_bounds__(GTHREADS, 2) attn_generic_kernel(const __grid_
   int n_desc = 0;
   int64_t base_row = 0;
   if (!CALIB) {
-    PlanView pv(p.seqs[seq].plan);
-    const int u = (p.step * p.L + p.layer) * p.H;
-    head = pv.order()[u + blockIdx.z];                   // heavy heads first
-    descs = pv.descs() + pv.attn_begin()[u + head];
-    n_desc = pv.attn_cnt()[u + head];
+    if (p.table_heads > 0) {
+      // one schedule for the whole call: the host listed, per head in dispatch order, where its descriptors
+      // start, so the first key tile is two dependent loads away instead of four
+      head = p.table_head[blockIdx.z];
+      descs = reinterpret_cast<const int2*>(p.seqs[seq].plan + p.table_desc_begin[blockIdx.z]);
+      n_desc = p.table_ndesc[blockIdx.z];
+    } else {
+      PlanView pv(p.seqs[seq].plan);
+      const int u = (p.step * p.L + p.layer) * p.H;
+      head = pv.order()[u + blockIdx.z];                   // heavy heads first
+      descs = pv.descs() + pv.attn_begin()[u + head];
+      n_desc = pv.attn_cnt()[u + head];
+    }
     base_row = p.seqs[seq].base_row;
   }
   const int n_own_tiles = (p.n_own + GN - 1) / GN;
@@ -97,12 +107,14 @@ __global__ void __launch_bounds__(GTHREADS, 2) attn_generic_kernel(const __grid_
   const __nv_bfloat16* kown = p.k_new + seq * p.kv_seq + head * p.kv_head;
   const __nv_bfloat16* vown = p.v_new ? p.v_new + seq * p.kv_seq + head * p.kv_head : nullptr;
 
+  // descriptors are fetched one tile ahead of the copy they steer: `dsc_next` belongs to the tile issued next
+  int2 dsc_next = n_desc > 0 ? descs[0] : make_int2(0, 0);
   auto issue_tile = [&](int j, int stage) {
     const __nv_bfloat16 *ks, *vs;
     int64_t stride;
     int nv;
     if (j < n_desc) {
-      int2 dsc = descs[j];
+      int2 dsc = dsc_next;
       int64_t row = base_row + dsc.x;
       ks = p.k_pool + row * D;
       vs = p.v_pool + row * D;
@@ -117,15 +129,18 @@ __global__ void __launch_bounds__(GTHREADS, 2) attn_generic_kernel(const __grid_
     }
     load_tile<D>(sbase + SM::K_OFF + stage * SM::TILE_BYTES, ks, stride, nv, tid);
     if (vs) load_tile<D>(sbase + SM::V_OFF + stage * SM::TILE_BYTES, vs, stride, nv, tid);
+    if (j + 1 < n_desc) dsc_next = descs[j + 1];
   };
 
-  // ---- prologue: Q tile and the first key tile
+  // ---- prologue: Q tile and the first GSTAGES - 1 key tiles, one copy group each (empty groups keep the count)
   {
     const __nv_bfloat16* qsrc = p.q + seq * p.q_seq + head * p.q_head + (int64_t)q0 * p.q_tok;
     load_tile<D>(sbase + SM::Q_OFF, qsrc, p.q_tok, min(GM, p.t_q - q0), tid);
     cp_async_commit();
-    issue_tile(0, 0);
-    cp_async_commit();
+    for (int j = 0; j < GSTAGES - 1; ++j) {
+      if (j < n_tiles) issue_tile(j, j);
+      cp_async_commit();
+    }
   }
   if (CALIB) {
     for (int i = tid; i < GM * HEATKV_MAX_K; i += GTHREADS) {
@@ -133,7 +148,7 @@ __global__ void __launch_bounds__(GTHREADS, 2) attn_generic_kernel(const __grid_
       seg_ref[i] = -INFINITY;
     }
   }
-  cp_async_wait<1>();
+  cp_async_wait<GSTAGES - 1>();                        // Q has landed
   __syncthreads();
 
   uint32_t qf[D / 16][4];
@@ -151,10 +166,10 @@ __global__ void __launch_bounds__(GTHREADS, 2) attn_generic_kernel(const __grid_
   float l_run[2] = {0.f, 0.f};
 
   for (int j = 0; j < n_tiles; ++j) {
-    const int stage = j & 1;
-    cp_async_wait<0>();
-    __syncthreads();                                   // tile j landed; everyone left tile j-1
-    if (j + 1 < n_tiles) issue_tile(j + 1, stage ^ 1);
+    const int stage = j % GSTAGES;
+    cp_async_wait<GSTAGES - 2>();                      // all groups but the newest GSTAGES - 2: tile j is among them
+    __syncthreads();                                   // tile j landed for everyone; everyone left tile j-1
+    if (j + GSTAGES - 1 < n_tiles) issue_tile(j + GSTAGES - 1, (j + GSTAGES - 1) % GSTAGES);   // into tile j-1's stage
     cp_async_commit();
 
     // tile attributes (warp-uniform)
@@ -375,14 +390,15 @@ __global__ void reduce_partials_kernel(const float* partials, float* beta_row, i
 template <int D, bool CALIB>
 static cudaError_t launch_one(const AttnParams& p, int n_seq, cudaStream_t stream) {
   auto kern = attn_generic_kernel<D, CALIB>;
+  constexpr int bytes = CALIB ? GenericSmem<D>::BYTES : GenericSmem<D>::ATTN_BYTES;
   static bool configured = false;
   if (!configured) {
-    cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, GenericSmem<D>::BYTES);
+    cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, bytes);
     if (e != cudaSuccess) return e;
     configured = true;
   }
   dim3 grid((p.t_q + GM - 1) / GM + (CALIB ? 0 : p.append_tiles), CALIB ? p.H : n_seq, CALIB ? n_seq : p.H);
-  kern<<<grid, GTHREADS, GenericSmem<D>::BYTES, stream>>>(p);
+  kern<<<grid, GTHREADS, bytes, stream>>>(p);
   return cudaGetLastError();
 }
 

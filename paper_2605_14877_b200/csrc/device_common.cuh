@@ -52,6 +52,10 @@ struct AttnParams {
   int32_t attn_items, store_items;  // tensor-memory kernel: attention work items; cache-update items (destination half-tiles)
   float* split_partials;          // [n_seq * slots_per_seq][SPLIT_SLOT_FLOATS]
   uint32_t* split_counters;       // [n_seq * ctrs_per_seq], zero between launches
+  // generic kernel, with table_heads > 0: per head in dispatch order, the half-tile descriptors of its visible
+  // prior keys (count, and word offset of the first in the plan blob)
+  int16_t table_ndesc[64];
+  int32_t table_desc_begin[64];
 };
 
 struct CopyParams {
