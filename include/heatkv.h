@@ -22,6 +22,10 @@
  *  - Every function returns HEATKV_OK (0) or a negative heatkv_status.  Nothing throws or
  *    aborts across this boundary; a call that fails leaves cache and context unchanged.
  *  - A context is not thread-safe; use one context per thread or lock around it.
+ *  - The kernels of one context share work counters and scratch inside its arena, so they must
+ *    not overlap on the GPU: enqueue a context's calls on one stream, or order the streams
+ *    with events.  After HEATKV_ERR_DEVICE_TIMEOUT (heatkv_device_status) a context stays in
+ *    that state; destroy it and create a new one.
  */
 #ifndef HEATKV_H_
 #define HEATKV_H_
