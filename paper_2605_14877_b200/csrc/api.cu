@@ -335,7 +335,7 @@ void fill_head_table(heatkv_ctx* ctx, const int* seq_ids, int n_seq, int step, i
 // cut further so that the last round of items fills the SMs.  It is cached per (schedule, step, layer, batch
 // size).  Calls that mix schedules use one longest run for all of them.
 void choose_split(heatkv_ctx* ctx, const int* seq_ids, int n_seq, int step, int layer, AttnParams* p) {
-  constexpr int MIN_PIECE = 6;                              // pieces about as short as the fixed cost never pay
+  constexpr int MIN_PIECE = 4;                              // shorter pieces measured slower (their fixed cost dominates)
   const int n_qp = (p->t_q + 255) / 256, own_slots = (p->n_own + HEATKV_PAGE_TOKENS - 1) / HEATKV_PAGE_TOKENS;
   const PlanEntry& pe0 = *ctx->plans[ctx->seqs[seq_ids[0]].plan];
   bool one_plan = pe0.sched.H <= 64;
