@@ -332,6 +332,50 @@ def run_few_heads_workload(args):
     print(json.dumps({"workload": "few_heads_key_range_splitting", "runs": rows}), flush=True)
 
 
+def run_head_dim_64_workload(args):
+    """A layer of the same width as the headline's with heads of 64 instead of 128 dimensions (32 heads, 13
+    scales, batch 2, budget 1/20; not the headline line): every sweep timed call by call on the tcgen05 kernel's
+    head_dim-64 instantiation (kernel auto) and on the warp-level MMA kernel alone."""
+    import paper_2605_14877_b200 as hk
+    from paper_2605_14877_b200.sweep import Session
+    torch.cuda.set_device(0)
+    sh = W.Shape("width2048_d64", L=1, H=32, d=64, sides=W.SIDES_13, n_seq=2, s=3)
+    scores = W.synthetic_scas(sh, 0)
+    q, k, v = W.qkv_layer(sh, 0, 0, device="cuda")
+    c = [0] + sh.c
+    qs, ks, vs = ([x[:, :, c[i]:c[i + 1]].contiguous() for i in range(sh.K)] for x in (q, k, v))
+    outs = [torch.zeros_like(x) for x in qs]
+    flush = torch.empty(256 << 20, dtype=torch.uint8, device="cuda")
+    res = {"workload": "head_dim_64_layer", "H": sh.H, "d": sh.d, "n_seq": sh.n_seq, "budget": B_BUDGET}
+    for name, kernel in (("auto", hk.KERNEL_AUTO), ("generic", hk.KERNEL_GENERIC)):
+        ses = Session(sh.L, sh.H, sh.d, sh.t, sh.s, pool_rows=2 * sh.n_seq * sh.H * (sh.c[-2] + 64 * sh.K), kernel=kernel)
+        sch = ses.schedule(scas=scores, b=B_BUDGET)
+        am, _, _, _ = hk.heatkv_schedule_masks(sch, sh.K, sh.L, sh.H)
+        flops = attention_flops(sh, am, sh.n_seq)
+        ms, reps = np.zeros(sh.K), max(3, min(args.steps, 20))
+        for rep in range(reps + 2):
+            ids = [hk.heatkv_seq_open(ses.ctx, sch) for _ in range(sh.n_seq)]
+            for step in range(sh.K):
+                ses.pre_step(ids, step)
+                flush.fill_(1)
+                e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+                e0.record()
+                hk.heatkv_attention_append(ses.ctx, ids, 0, step, qs[step], ks[step], vs[step], None, None, outs[step])
+                e1.record()
+                torch.cuda.synchronize()
+                if rep >= 2:
+                    ms[step] += e0.elapsed_time(e1) / reps
+            for i in ids:
+                hk.heatkv_seq_close(ses.ctx, i)
+        assert hk.heatkv_device_status(ses.ctx) == 0
+        res[name + "_ms_per_scale"] = [round(float(x), 4) for x in ms]
+        res[name + "_sum_ms"] = round(float(ms.sum()), 4)
+        res[name + "_tflops_largest"] = round(flops[sh.K - 1] / (float(ms[sh.K - 1]) * 1e-3) / 1e12, 1)
+        hk.heatkv_schedule_free(sch)
+        ses.close()
+    print(json.dumps(res), flush=True)
+
+
 def run_stability_workload(args):
     """Synthetic analogue of the paper's S-CAS stability study (not the headline line): the S-CAS head
     ordering is computed from 10 independently seeded calibration sets (4 sequences each) of a 4-layer x
@@ -495,7 +539,7 @@ def main():
     ap.add_argument("--calls", default="fused", choices=["fused", "separate"],
                     help="fused: heatkv_attention_append (one launch per step in the paged layout); separate: "
                          "heatkv_scale_attention followed by heatkv_append_compact")
-    ap.add_argument("--workload", default="config2", choices=["config2", "cache", "full", "larger", "serving", "fewheads", "stability"],
+    ap.add_argument("--workload", default="config2", choices=["config2", "cache", "full", "larger", "serving", "fewheads", "stability", "d64"],
                     help="config2: the headline line; cache: append / compaction GB/s at a saturating shape; "
                          "full / larger / serving: whole-model sweeps of the other workloads; fewheads: key-range "
                          "splitting on launches with few (sequence, head) units; stability: S-CAS rank spread "
@@ -518,6 +562,9 @@ def main():
     if args.workload == "stability":
         if rank == 0:
             run_stability_workload(args)
+        return
+    if args.workload == "d64":
+        run_head_dim_64_workload(args)
         return
     if args.workload == "fewheads":
         if rank == 0:

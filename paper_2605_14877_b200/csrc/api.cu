@@ -22,7 +22,7 @@ void tc_destroy(TcState* st);
 bool tc_supported(const TcState* st, const AttnParams& p, int d, int n_seq, bool calib);
 cudaError_t launch_attn_tc(TcState* st, const AttnParams& p, int d, int n_seq, bool calib, cudaStream_t stream,
                            int* launches);
-int tc_split_slot_floats();
+int tc_split_slot_floats(int d);
 struct CalibTcState;
 uint64_t calib_tc_desc_bytes(const heatkv_config& cfg);
 int calib_tc_create(const heatkv_config& cfg, void* dev_table, cudaStream_t stream, CalibTcState** out);
@@ -486,7 +486,7 @@ int heatkv_create(const heatkv_config* cfg, void* stream_, heatkv_ctx** out) {
   ctx->k_pool = reinterpret_cast<__nv_bfloat16*>(ctx->meta + meta + scratch);
   {   // scratch region: arrival counters first (kept zero between launches), then the partial-result slots
     const uint64_t ctr_bytes = std::min<uint64_t>(scratch / 4, 256u << 10) / 1024 * 1024;
-    const uint64_t slot_bytes = (uint64_t)tc_split_slot_floats() * 4;
+    const uint64_t slot_bytes = (uint64_t)tc_split_slot_floats(cfg->d) * 4;
     ctx->split_counters = reinterpret_cast<uint32_t*>(ctx->meta + meta);
     ctx->split_ctrs = ctr_bytes / 4;
     ctx->split_partials = reinterpret_cast<float*>(ctx->meta + meta + ctr_bytes);

@@ -31,7 +31,6 @@ namespace heatkv {
 
 namespace tc {
 
-constexpr int D = 128;
 constexpr int BM = 128;                 // rows per Q tile
 constexpr int BN = 128;                 // keys per tile (two 64-row half-tiles)
 constexpr int HALF = 64;
@@ -45,19 +44,29 @@ constexpr int REGS_SMALL = 72;
 constexpr int REGS_SOFTMAX = 216;
 static_assert(128 * REGS_SMALL + 256 * REGS_SOFTMAX <= THREADS * REGS_LAUNCH, "register hand-over exceeds the CTA's allocation");
 constexpr uint32_t HALF_COLS_BYTES = 128 * 128;        // one 64-column half of a 128-row tile: 16 KB
-constexpr uint32_t TILE_BYTES = 2 * HALF_COLS_BYTES;   // 32 KB
 constexpr uint32_t SLOT_BYTES = HALF * 128;            // 64 rows x 128 B inside one column half
 constexpr uint32_t STAGE_BYTES = 4096;                 // per softmax warp: two buffers of 32 rows x 64 B for the output rows
 
-// shared memory map (bytes from a 1024-aligned base)
-constexpr uint32_t SM_Q = 0;                                   // 2 tiles
-constexpr uint32_t SM_K = SM_Q + 2 * TILE_BYTES;               // KV_STAGES tiles
-constexpr uint32_t SM_V = SM_K + KV_STAGES * TILE_BYTES;       // KV_STAGES tiles
-constexpr uint32_t SM_OUT = SM_V + KV_STAGES * TILE_BYTES;     // output staging of the eight softmax warps
-constexpr uint32_t SM_BAR = SM_OUT + 8 * STAGE_BYTES;          // barriers + scalars + item ring
-constexpr uint32_t SM_TOTAL = SM_BAR + 512;
-constexpr uint32_t SM_ALLOC = SM_TOTAL + 1024;                 // slack for manual alignment
-static_assert(SM_ALLOC <= 227 * 1024, "shared memory of one CTA");
+// Sizes that follow the head dimension D (64 or 128): a 128-row tile is D / 64 column halves of 16 KB.
+template <int D>
+struct Layout {
+  static_assert(D == 64 || D == 128, "head dimension");
+  static constexpr int NCH = D / 64;                             // 64-column halves per row
+  static constexpr uint32_t TILE_BYTES = NCH * HALF_COLS_BYTES;  // 16 or 32 KB
+  // shared memory map (bytes from a 1024-aligned base)
+  static constexpr uint32_t SM_Q = 0;                                   // 2 tiles
+  static constexpr uint32_t SM_K = SM_Q + 2 * TILE_BYTES;               // KV_STAGES tiles
+  static constexpr uint32_t SM_V = SM_K + KV_STAGES * TILE_BYTES;       // KV_STAGES tiles
+  static constexpr uint32_t SM_OUT = SM_V + KV_STAGES * TILE_BYTES;     // output staging of the eight softmax warps
+  static constexpr uint32_t SM_BAR = SM_OUT + 8 * STAGE_BYTES;          // barriers + scalars + item ring
+  static constexpr uint32_t SM_TOTAL = SM_BAR + 512;
+  static constexpr uint32_t SM_ALLOC = SM_TOTAL + 1024;                 // slack for manual alignment
+  static_assert(SM_ALLOC <= 227 * 1024, "shared memory of one CTA");
+  // One partial result of a split head: unnormalised O of both query tiles (fp32, groups of four columns
+  // outermost so that a warp's 32 rows touch consecutive 16-byte words), then the rows' running references
+  // and row sums.
+  static constexpr int SPLIT_SLOT_FLOATS = 2 * BM * D + 2 * 2 * BM;
+};
 
 // barrier slots (8 bytes each) inside SM_BAR
 enum Bar : uint32_t {
@@ -70,16 +79,12 @@ enum Bar : uint32_t {
   ITEM_FULL = 20, ITEM_EMPTY = 22,  // +ring entry; EMPTY takes one arrival from the MMA warp and each softmax warp
   N_BARS = 24
 };
-constexpr uint32_t SM_TMEM_PTR = SM_BAR + N_BARS * 8;
-constexpr uint32_t SM_ABORT = SM_TMEM_PTR + 4;
-constexpr uint32_t SM_RING = SM_BAR + 256;                     // 2 entries x int32[16]
+constexpr uint32_t BAR_TMEM_PTR = N_BARS * 8;                  // offsets inside the barrier region
+constexpr uint32_t BAR_ABORT = BAR_TMEM_PTR + 4;
+constexpr uint32_t BAR_RING = 256;                             // 2 entries x int32[16]
 enum ItemKind : int { ATTENTION = 0, STOP = 2, NOTHING = 3 };
 // ring entry words
 enum ItemWord : int { W_KIND = 0, W_HEAD, W_SEQ, W_TILES, W_NSPLIT, W_SUB, W_SLOT, W_CTR, W_DESC, W_NDESC };
-// One partial result of a split head: unnormalised O of both query tiles (fp32, groups of four columns
-// outermost so that a warp's 32 rows touch consecutive 16-byte words), then the rows' running references
-// and row sums.
-constexpr int SPLIT_SLOT_FLOATS = 2 * BM * D + 2 * 2 * BM;
 constexpr int WORK_COUNTER_WORD = 16;                          // word of the status region that hands out the attention items
 constexpr int STORE_COUNTER_WORD = 17;                         // ... and the cache-update items
 
@@ -142,8 +147,15 @@ __device__ __forceinline__ Item read_item(const volatile int32_t* ring, const At
   return it;
 }
 
+template <int D>
 __global__ void __launch_bounds__(THREADS, 1)
 attn_tc_kernel(const __grid_constant__ AttnParams p, const __grid_constant__ Maps maps) {
+  using L = Layout<D>;
+  constexpr int NCH = L::NCH;
+  constexpr uint32_t TILE_BYTES = L::TILE_BYTES, SM_Q = L::SM_Q, SM_K = L::SM_K, SM_V = L::SM_V, SM_OUT = L::SM_OUT,
+                     SM_BAR = L::SM_BAR, SM_TMEM_PTR = L::SM_BAR + BAR_TMEM_PTR, SM_ABORT = L::SM_BAR + BAR_ABORT,
+                     SM_RING = L::SM_BAR + BAR_RING;
+  constexpr int SPLIT_SLOT_FLOATS = L::SPLIT_SLOT_FLOATS;
   extern __shared__ unsigned char smem_raw[];
   const uint32_t raw = smem_u32(smem_raw);
   const uint32_t sbase = (raw + 1023u) & ~1023u;
@@ -302,7 +314,7 @@ attn_tc_kernel(const __grid_constant__ AttnParams p, const __grid_constant__ Map
         if (leader) {
           mbar_expect_tx(bar(K_FULL + st), TILE_BYTES);
           for (int hf = 0; hf < 2; ++hf)
-            for (int ch = 0; ch < 2; ++ch) {
+            for (int ch = 0; ch < NCH; ++ch) {
               uint32_t dst = sbase + SM_K + st * TILE_BYTES + ch * HALF_COLS_BYTES + hf * SLOT_BYTES;
               if (sl[hf].pool_row >= 0) tma_load_2d(dst, &maps.k_pool, ch * 64, sl[hf].pool_row, bar(K_FULL + st));
               else tma_load_4d(dst, &maps.k_own, ch * 64, -sl[hf].pool_row - 1, im.head, seq, bar(K_FULL + st));
@@ -320,7 +332,7 @@ attn_tc_kernel(const __grid_constant__ AttnParams p, const __grid_constant__ Map
             ++iq[x];
             if (leader) {
               mbar_expect_tx(bar(Q_FULL + x), TILE_BYTES);
-              for (int ch = 0; ch < 2; ++ch)
+              for (int ch = 0; ch < NCH; ++ch)
                 for (int hf = 0; hf < 2; ++hf)
                   tma_load_4d(sbase + SM_Q + x * TILE_BYTES + ch * HALF_COLS_BYTES + hf * SLOT_BYTES, &maps.q, ch * 64,
                               im.q0 + x * BM + hf * HALF, im.head, seq, bar(Q_FULL + x));
@@ -335,7 +347,7 @@ attn_tc_kernel(const __grid_constant__ AttnParams p, const __grid_constant__ Map
         if (leader) {
           mbar_expect_tx(bar(V_FULL + st), TILE_BYTES);
           for (int hf = 0; hf < 2; ++hf)
-            for (int ch = 0; ch < 2; ++ch) {
+            for (int ch = 0; ch < NCH; ++ch) {
               uint32_t dst = sbase + SM_V + st * TILE_BYTES + ch * HALF_COLS_BYTES + hf * SLOT_BYTES;
               if (sl[hf].pool_row >= 0) tma_load_2d(dst, &maps.v_pool, ch * 64, sl[hf].pool_row, bar(V_FULL + st));
               else tma_load_4d(dst, &maps.v_own, ch * 64, -sl[hf].pool_row - 1, im.head, seq, bar(V_FULL + st));
@@ -575,7 +587,7 @@ attn_tc_kernel(const __grid_constant__ AttnParams p, const __grid_constant__ Map
               tc_fence_after();
               const float f = grow ? exp2f(m_ref - m_new) : 1.f;
 #pragma unroll
-              for (int c = 0; c < 4; ++c) {
+              for (int c = 0; c < D / 32; ++c) {
                 uint32_t r[32];
                 tmem_ld32(t_o + c * 32, r);
                 tmem_wait_ld();
@@ -664,11 +676,9 @@ attn_tc_kernel(const __grid_constant__ AttnParams p, const __grid_constant__ Map
             tc_fence_after();
             const float inv = 1.f / l_sum;
             // the whole row of O in one go, so the four groups' conversions and stores overlap
-            uint32_t o0[32], o1[32], o2[32], o3[32];
-            tmem_ld32(t_o, o0);
-            tmem_ld32(t_o + 32, o1);
-            tmem_ld32(t_o + 64, o2);
-            tmem_ld32(t_o + 96, o3);
+            uint32_t o[D / 32][32];
+#pragma unroll
+            for (int c = 0; c < D / 32; ++c) tmem_ld32(t_o + c * 32, o[c]);
             tmem_wait_ld();
             auto out_group = [&](const uint32_t (&r)[32], int c) {
               float acc[32];
@@ -676,10 +686,8 @@ attn_tc_kernel(const __grid_constant__ AttnParams p, const __grid_constant__ Map
               for (int i = 0; i < 32; ++i) acc[i] = __uint_as_float(r[i]);
               store_rows(acc, inv, c);
             };
-            out_group(o0, 0);
-            out_group(o1, 1);
-            out_group(o2, 2);
-            out_group(o3, 3);
+#pragma unroll
+            for (int c = 0; c < D / 32; ++c) out_group(o[c], c);
           } else if (ok) {
             // A piece of a split head: publish the unnormalised O of this row with its reference and row
             // sum; the warp that arrives last at the counter of these 32 rows merges
@@ -690,7 +698,7 @@ attn_tc_kernel(const __grid_constant__ AttnParams p, const __grid_constant__ Map
             float* slot_own = slots + (int64_t)im.sub * SPLIT_SLOT_FLOATS;
             int4* ocol = reinterpret_cast<int4*>(slot_own) + x * BM + row;
 #pragma unroll 1
-            for (int c = 0; c < 4; ++c) {
+            for (int c = 0; c < D / 32; ++c) {
               uint32_t r[32];
               tmem_ld32(t_o + c * 32, r);
               tmem_wait_ld();
@@ -727,7 +735,7 @@ attn_tc_kernel(const __grid_constant__ AttnParams p, const __grid_constant__ Map
               }
               const float inv = 1.f / l_all;
 #pragma unroll 1
-              for (int c = 0; c < 4; ++c) {
+              for (int c = 0; c < D / 32; ++c) {
                 uint32_t r[32];
                 tmem_ld32(t_o + c * 32, r);
                 tmem_wait_ld();
@@ -776,14 +784,15 @@ struct TcState {
   PFN_cuTensorMapEncodeTiled_v12000 encode = nullptr;
   CUtensorMap k_pool, v_pool;
   int n_sm = 148;
+  int d = 0;                 // head dimension of the context (64 or 128)
   bool ready = false;
 };
 
 namespace {
 
 bool encode_2d(TcState* st, CUtensorMap* m, void* base, uint64_t rows) {
-  cuuint64_t dims[2] = {(cuuint64_t)tc::D, (cuuint64_t)rows};
-  cuuint64_t strides[1] = {(cuuint64_t)tc::D * 2};
+  cuuint64_t dims[2] = {(cuuint64_t)st->d, (cuuint64_t)rows};
+  cuuint64_t strides[1] = {(cuuint64_t)st->d * 2};
   cuuint32_t box[2] = {64, (cuuint32_t)tc::HALF};
   cuuint32_t estr[2] = {1, 1};
   return st->encode(m, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, base, dims, strides, box, estr,
@@ -794,7 +803,7 @@ bool encode_2d(TcState* st, CUtensorMap* m, void* base, uint64_t rows) {
 // [n_seq, H, t, d] view with element strides -> 4-D map (d, token, head, sequence)
 bool encode_4d(TcState* st, CUtensorMap* m, const void* base, int t, int H, int n_seq, int64_t s_tok, int64_t s_head,
                int64_t s_seq) {
-  cuuint64_t dims[4] = {(cuuint64_t)tc::D, (cuuint64_t)t, (cuuint64_t)H, (cuuint64_t)n_seq};
+  cuuint64_t dims[4] = {(cuuint64_t)st->d, (cuuint64_t)t, (cuuint64_t)H, (cuuint64_t)n_seq};
   // a stride of 0 is not encodable; a dimension of extent 1 may carry any positive stride
   auto fix = [](int64_t s) { return (cuuint64_t)((s > 0 ? s : 8) * 2); };
   cuuint64_t strides[3] = {fix(s_tok), fix(s_head), fix(s_seq)};
@@ -812,7 +821,8 @@ int tc_create(const heatkv_config& cfg, void* k_pool, void* v_pool, uint64_t poo
   TcState* st = new (std::nothrow) TcState;
   if (!st) return HEATKV_ERR_HOST_MEMORY;
   *out = st;
-  if (cfg.d != tc::D) return HEATKV_OK;                 // only head_dim 128 runs on this path
+  if (cfg.d != 64 && cfg.d != 128) return HEATKV_OK;    // other head dimensions run on the generic kernel only
+  st->d = cfg.d;
   void* fn = nullptr;
   cudaDriverEntryPointQueryResult qres;
   if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &fn, cudaEnableDefault, &qres) != cudaSuccess ||
@@ -823,14 +833,15 @@ int tc_create(const heatkv_config& cfg, void* k_pool, void* v_pool, uint64_t poo
   st->encode = reinterpret_cast<PFN_cuTensorMapEncodeTiled_v12000>(fn);
   if (!encode_2d(st, &st->k_pool, k_pool, pool_rows) || !encode_2d(st, &st->v_pool, v_pool, pool_rows))
     return HEATKV_OK;
-  if (cudaFuncSetAttribute(tc::attn_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)tc::SM_ALLOC) !=
-      cudaSuccess) {
+  const void* kern = cfg.d == 128 ? (const void*)tc::attn_tc_kernel<128> : (const void*)tc::attn_tc_kernel<64>;
+  const int smem = cfg.d == 128 ? (int)tc::Layout<128>::SM_ALLOC : (int)tc::Layout<64>::SM_ALLOC;
+  if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, smem) != cudaSuccess) {
     cudaGetLastError();
     return HEATKV_OK;
   }
   // the register hand-over inside the kernel must fit in what the launch really allocates
   cudaFuncAttributes attr;
-  if (cudaFuncGetAttributes(&attr, tc::attn_tc_kernel) != cudaSuccess) {
+  if (cudaFuncGetAttributes(&attr, kern) != cudaSuccess) {
     cudaGetLastError();
     return HEATKV_OK;
   }
@@ -845,10 +856,10 @@ int tc_create(const heatkv_config& cfg, void* k_pool, void* v_pool, uint64_t poo
 
 void tc_destroy(TcState* st) { delete st; }
 
-int tc_split_slot_floats() { return tc::SPLIT_SLOT_FLOATS; }
+int tc_split_slot_floats(int d) { return d == 64 ? tc::Layout<64>::SPLIT_SLOT_FLOATS : tc::Layout<128>::SPLIT_SLOT_FLOATS; }
 
 bool tc_supported(const TcState* st, const AttnParams& p, int d, int n_seq, bool calib) {
-  if (!st || !st->ready || calib || d != tc::D || n_seq > 65535) return false;
+  if (!st || !st->ready || calib || d != st->d || n_seq > 65535) return false;
   // TMA needs 16-byte aligned bases (checked by the caller) and strides that are multiples of 16 bytes
   const int64_t s[6] = {p.q_seq, p.q_head, p.q_tok, p.kv_seq, p.kv_head, p.kv_tok};
   for (int64_t v : s)
@@ -872,7 +883,8 @@ cudaError_t launch_attn_tc(TcState* st, const AttnParams& p, int d, int n_seq, b
   q.attn_items = p.items_per_seq * n_seq;
   q.store_items = p.append_tiles * p.H * n_seq;
   dim3 grid((unsigned)std::min(q.attn_items, st->n_sm));
-  tc::attn_tc_kernel<<<grid, tc::THREADS, tc::SM_ALLOC, stream>>>(q, maps);
+  if (st->d == 128) tc::attn_tc_kernel<128><<<grid, tc::THREADS, tc::Layout<128>::SM_ALLOC, stream>>>(q, maps);
+  else tc::attn_tc_kernel<64><<<grid, tc::THREADS, tc::Layout<64>::SM_ALLOC, stream>>>(q, maps);
   *launches = 1;
   return cudaGetLastError();
 }

@@ -153,6 +153,24 @@ def test_tensor_memory_kernel_mid_config(hk, layout):
                      kernel=hk.KERNEL_TCGEN05)
 
 
+@pytest.mark.parametrize("layout", [0, 1], ids=["ragged", "paged"])
+def test_tensor_memory_kernel_head_dim_64(hk, layout):
+    """The tcgen05 kernel's head_dim-64 instantiation (one 64-column half per row, N = 64 PV products) on every
+    step of a mid workload with bias, cache update in the same call; and a split launch (few heads, long ranges)."""
+    sh = W.Shape("mid64", L=2, H=4, d=64, sides=W.SIDES_13[:11], n_seq=2, s=3)
+    scores = W.synthetic_scas(sh, 5)
+    ref = O.heatkv_schedule(scores, 0.15, sh.s, sh.sides)
+    bias = W.seg_bias_prior_lognormal(sh, 4)
+    _run_full_parity(hk, sh, ref, lambda ses: ses.schedule(scas=scores, b=0.15), layout, bias=bias,
+                     kernel=hk.KERNEL_TCGEN05, fused=True)
+    if layout == 1:
+        sh2 = W.Shape("split64", L=1, H=3, d=64, sides=W.SIDES_13[:12], n_seq=2, s=3)
+        scores2 = W.synthetic_scas(sh2, 3)
+        ref2 = O.heatkv_schedule(scores2, 0.6, sh2.s, sh2.sides)
+        _run_full_parity(hk, sh2, ref2, lambda ses: ses.schedule(scas=scores2, b=0.6), hk.LAYOUT_PAGED,
+                         kernel=hk.KERNEL_AUTO, check_cache=False)
+
+
 def test_tensor_memory_kernel_full_cache(hk):
     """b = 1: long page tables (up to 4121 prior keys), tcgen05 kernel, no bias."""
     sh = W.Shape("full128", L=1, H=2, d=128, sides=W.SIDES_13[:12], n_seq=1, s=3)
