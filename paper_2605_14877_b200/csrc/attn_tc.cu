@@ -1,4 +1,4 @@
-// Tensor-memory attention kernel for the large scale steps (head_dim 128).
+// Tensor-memory attention kernel for the large scale steps (head_dim 128 or 64).
 //
 // The launch is a list of work items handed out through a counter: one CTA per SM stays resident and takes
 // item after item, so the loads and first products of the next item run under the epilogue of the current
