@@ -27,7 +27,7 @@ namespace calib {
 
 using namespace tc;
 
-constexpr int D = 128;
+constexpr int D_MAX = 128;               // the shared-memory map is sized for 128-wide heads; 64-wide ones use half of each tile
 constexpr int BM = 128;                 // rows per Q tile
 constexpr int BN = 128;                 // keys per tile (two 64-row half-tiles)
 constexpr int HALF = 64;
@@ -76,9 +76,13 @@ __device__ __forceinline__ HalfTile get_half(int i, const int2* descs, int n_slo
   return h;
 }
 
+template <int D>
 __global__ void __launch_bounds__(THREADS, 1)
 calib_tc_kernel(const __grid_constant__ AttnParams p, const __grid_constant__ Maps maps, const int2* __restrict__ descs,
                 int n_slots) {
+  static_assert(D == 64 || D == 128, "head dimension");
+  constexpr int NCH = D / 64;                               // 64-column halves per row
+  constexpr uint32_t LOAD_BYTES = NCH * HALF_COLS_BYTES;    // bytes one tile's copies deliver
   extern __shared__ unsigned char smem_raw[];
   const uint32_t raw = smem_u32(smem_raw);
   const uint32_t sbase = (raw + 1023u) & ~1023u;
@@ -130,8 +134,8 @@ calib_tc_kernel(const __grid_constant__ AttnParams p, const __grid_constant__ Ma
       uint32_t par[K_STAGES] = {0, 0, 0, 0};
       if (leader) {
         for (int x = 0; x < nq; ++x) {
-          mbar_expect_tx(bar(Q_FULL + x), TILE_BYTES);
-          for (int ch = 0; ch < 2; ++ch)
+          mbar_expect_tx(bar(Q_FULL + x), LOAD_BYTES);
+          for (int ch = 0; ch < NCH; ++ch)
             for (int hf = 0; hf < 2; ++hf)
               tma_load_4d(sbase + SM_Q + x * TILE_BYTES + ch * HALF_COLS_BYTES + hf * SLOT_BYTES, &maps.q, ch * 64,
                           q0 + x * BM + hf * HALF, head, seq, bar(Q_FULL + x));
@@ -147,9 +151,9 @@ calib_tc_kernel(const __grid_constant__ AttnParams p, const __grid_constant__ Ma
         armed |= 1u << st;
         par[st] = use & 1;
         if (leader) {
-          mbar_expect_tx(bar(K_FULL + st), TILE_BYTES);
+          mbar_expect_tx(bar(K_FULL + st), LOAD_BYTES);
           for (int hf = 0; hf < 2; ++hf)
-            for (int ch = 0; ch < 2; ++ch)
+            for (int ch = 0; ch < NCH; ++ch)
               tma_load_4d(sbase + SM_K + st * TILE_BYTES + ch * HALF_COLS_BYTES + hf * SLOT_BYTES, &maps.k, ch * 64,
                           hf == 0 ? h0.row : h1.row, head, seq, bar(K_FULL + st));
         }
@@ -337,6 +341,7 @@ struct CalibTcState {
   std::vector<int2> host_descs;          // all steps, concatenated (kept alive for the upload)
   std::vector<int> first, count;         // per step
   const int2* dev_descs = nullptr;
+  int d = 0;                             // head dimension of the context (64 or 128)
   bool ready = false;
 };
 
@@ -353,7 +358,8 @@ int calib_tc_create(const heatkv_config& cfg, void* dev_table, cudaStream_t stre
   CalibTcState* st = new (std::nothrow) CalibTcState;
   if (!st) return HEATKV_ERR_HOST_MEMORY;
   *out = st;
-  if (cfg.d != calib::D || !dev_table) return HEATKV_OK;       // only head_dim 128 runs on this path
+  if ((cfg.d != 64 && cfg.d != 128) || !dev_table) return HEATKV_OK;   // other head dimensions: generic kernel only
+  st->d = cfg.d;
   void* fn = nullptr;
   cudaDriverEntryPointQueryResult qres;
   if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &fn, cudaEnableDefault, &qres) != cudaSuccess ||
@@ -384,13 +390,13 @@ int calib_tc_create(const heatkv_config& cfg, void* dev_table, cudaStream_t stre
   // later calls may come on other streams: the table must be in place before create returns
   if (cudaStreamSynchronize(stream) != cudaSuccess) return HEATKV_ERR_CUDA;
   st->dev_descs = static_cast<const int2*>(dev_table);
-  if (cudaFuncSetAttribute(calib::calib_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)calib::SM_ALLOC) !=
-      cudaSuccess) {
+  const void* kern = cfg.d == 128 ? (const void*)calib::calib_tc_kernel<128> : (const void*)calib::calib_tc_kernel<64>;
+  if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)calib::SM_ALLOC) != cudaSuccess) {
     cudaGetLastError();
     return HEATKV_OK;
   }
   cudaFuncAttributes attr;
-  if (cudaFuncGetAttributes(&attr, calib::calib_tc_kernel) != cudaSuccess) {
+  if (cudaFuncGetAttributes(&attr, kern) != cudaSuccess) {
     cudaGetLastError();
     return HEATKV_OK;
   }
@@ -403,7 +409,7 @@ int calib_tc_create(const heatkv_config& cfg, void* dev_table, cudaStream_t stre
 void calib_tc_destroy(CalibTcState* st) { delete st; }
 
 bool calib_tc_supported(const CalibTcState* st, const AttnParams& p, int d, int n_seq) {
-  if (!st || !st->ready || d != calib::D || n_seq > 65535 || p.H > 65535) return false;
+  if (!st || !st->ready || d != st->d || n_seq > 65535 || p.H > 65535) return false;
   const int64_t s[6] = {p.q_seq, p.q_head, p.q_tok, p.kv_seq, p.kv_head, p.kv_tok};
   for (int64_t v : s)
     if (v & 7) return false;
@@ -413,7 +419,7 @@ bool calib_tc_supported(const CalibTcState* st, const AttnParams& p, int d, int 
 namespace {
 bool encode_4d(CalibTcState* st, CUtensorMap* m, const void* base, int t, int H, int n_seq, int64_t s_tok, int64_t s_head,
                int64_t s_seq) {
-  cuuint64_t dims[4] = {(cuuint64_t)calib::D, (cuuint64_t)t, (cuuint64_t)H, (cuuint64_t)n_seq};
+  cuuint64_t dims[4] = {(cuuint64_t)st->d, (cuuint64_t)t, (cuuint64_t)H, (cuuint64_t)n_seq};
   auto fix = [](int64_t s) { return (cuuint64_t)((s > 0 ? s : 8) * 2); };
   cuuint64_t strides[3] = {fix(s_tok), fix(s_head), fix(s_seq)};
   cuuint32_t box[4] = {64, (cuuint32_t)calib::HALF, 1, 1};
@@ -430,8 +436,12 @@ cudaError_t launch_calib_tc(CalibTcState* st, const AttnParams& p, int n_seq, cu
       !encode_4d(st, &maps.k, p.k_new, p.n_own, p.H, n_seq, p.kv_tok, p.kv_head, p.kv_seq))
     return cudaErrorInvalidValue;
   dim3 grid((p.t_q + 2 * calib::BM - 1) / (2 * calib::BM), n_seq, p.H);
-  calib::calib_tc_kernel<<<grid, calib::THREADS, calib::SM_ALLOC, stream>>>(p, maps, st->dev_descs + st->first[p.step],
-                                                                            st->count[p.step]);
+  if (st->d == 128)
+    calib::calib_tc_kernel<128><<<grid, calib::THREADS, calib::SM_ALLOC, stream>>>(p, maps, st->dev_descs + st->first[p.step],
+                                                                                   st->count[p.step]);
+  else
+    calib::calib_tc_kernel<64><<<grid, calib::THREADS, calib::SM_ALLOC, stream>>>(p, maps, st->dev_descs + st->first[p.step],
+                                                                                  st->count[p.step]);
   return cudaGetLastError();
 }
 

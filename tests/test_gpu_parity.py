@@ -329,11 +329,13 @@ def test_calibration_mid_with_bias_and_output(hk):
             assert np.allclose(scas[l, h], O.scas(ref[l, h], sh.s), rtol=RTOL_BETA, atol=1e-9)
 
 
+@pytest.mark.parametrize("d", [128, 64], ids=["d128", "d64"])
 @pytest.mark.parametrize("with_bias", [False, True], ids=["plain", "bias"])
-def test_calibration_tensor_memory_kernel(hk, with_bias):
+def test_calibration_tensor_memory_kernel(hk, with_bias, d):
     """Every step forced through the tcgen05 calibration kernel: one-row tiles, ragged source-scale
-    borders inside key tiles (36, 144, 400 tokens), an odd number of half-tiles, two query tiles."""
-    sh = W.Shape("mid", L=2, H=3, d=128, sides=W.SIDES_13[:11], n_seq=2, s=3)
+    borders inside key tiles (36, 144, 400 tokens), an odd number of half-tiles, two query tiles; heads of
+    128 and of 64 dimensions."""
+    sh = W.Shape("mid", L=2, H=3, d=d, sides=W.SIDES_13[:11], n_seq=2, s=3)
     bias = W.seg_bias_prior_lognormal(sh, 8) if with_bias else None
     beta, scas, cas, ref = _calibrate(hk, sh, seeds=[5], bias=bias, kernel=hk.KERNEL_TCGEN05)
     mask = ref > 1e-5
