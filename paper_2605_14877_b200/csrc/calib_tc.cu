@@ -1,4 +1,4 @@
-// Tensor-memory calibration kernel (Sec. 3.1, Eq. 2) for the large scale steps (head_dim 128).
+// Tensor-memory calibration kernel (Sec. 3.1, Eq. 2) for the large scale steps (head_dim 128 or 64).
 //
 // beta[step][i] needs, for every query row of the step, the share of its softmax mass that falls on
 // the keys of source scale i.  Only S = Q K^T is a contraction here: there is no PV product and no
