@@ -246,6 +246,19 @@ int heatkv_attention_append(heatkv_ctx* ctx, const int* seq_ids /*HOST*/, int n_
 int heatkv_attention_split(heatkv_ctx* ctx, const int* seq_ids /*HOST*/, int n_seq, int layer, int step,
                            int32_t* split_tiles, int32_t* items);
 
+/* The search behind heatkv_attention_split, on its own (pure host code, needs no context and no GPU): given
+ * the key tiles (128 keys each) of the heads of one launch in dispatch order (descending), the query tile
+ * pairs per head (ceil(t_step / 256)), the sequences of the call and the SMs of the device, writes to
+ * pieces[0..n_heads) into how many equal pieces every head's key range is cut (1 = whole head).  per_head = 0
+ * restricts the choice to "no piece longer than some run", the rule a call that mixes schedules uses.
+ * max_slots / max_ctrs bound the partial-result slots and arrival counters the cut may use (what the
+ * context's scratch region holds).  The two optional outputs are the estimated makespans, in key tiles,
+ * of the launch with whole heads and with the chosen cut.  Errors: INVALID_ARG for non-positive sizes or
+ * tiles that are not sorted in descending order. */
+int heatkv_split_plan(const int32_t* tiles /*HOST*/, int n_heads, int n_qp, int n_seq, int n_sm, int per_head,
+                      uint64_t max_slots, uint64_t max_ctrs, int32_t* pieces /*HOST*/, double* makespan_whole,
+                      double* makespan_cut);
+
 /* Introspection (host state only unless noted). */
 int heatkv_cache_bytes(heatkv_ctx* ctx, int seq_id, uint64_t* actual, uint64_t* reserved);
 /* Global token indices c_{i-1}+j of the tokens head (layer, head) holds now; idx HOST with

@@ -9,7 +9,7 @@ HERE = os.path.dirname(os.path.abspath(__file__))
 ROOT = os.path.dirname(HERE)
 CSRC = os.path.join(HERE, "csrc")
 LIB = os.path.join(HERE, "libheatkv.so")
-SOURCES = ["schedule.cpp", "plan.cpp", "api.cu", "attn_generic.cu", "attn_tc.cu", "calib_tc.cu", "cache_kernels.cu"]
+SOURCES = ["schedule.cpp", "plan.cpp", "split.cpp", "api.cu", "attn_generic.cu", "attn_tc.cu", "calib_tc.cu", "cache_kernels.cu"]
 
 
 def _stale() -> bool:

@@ -100,13 +100,6 @@ inline bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 
 
 }  // namespace
 
-// How one attention launch cuts its heads: pieces per head in dispatch order; `lmax` > 0 when that is the
-// same as "no run longer than lmax tiles" (the rule a call with several schedules applies to all of them).
-struct SplitChoice {
-  std::vector<int> ns;
-  int lmax = 0;
-};
-
 struct heatkv_ctx {
   heatkv_config cfg;
   int c[HEATKV_MAX_K];
@@ -246,11 +239,6 @@ int gather_seqs(heatkv_ctx* ctx, const int* seq_ids, int n_seq, int layer, int s
 }
 
 // ---- key-range splitting of the tensor-memory attention kernel -----------------------------------------
-// Items of one sequence: count, partial slots, counters.
-struct SplitShape {
-  int items = 0, slots = 0, ctrs = 0;
-};
-
 // Key tiles of the heads of (step, layer), in the plan's dispatch order (descending key count).
 std::vector<int> ordered_tiles(const PlanEntry& pe, int step, int layer, int own_slots) {
   const Schedule& s = pe.sched;
@@ -261,52 +249,6 @@ std::vector<int> ordered_tiles(const PlanEntry& pe, int step, int layer, int own
   std::vector<int> t(s.H);
   for (int i = 0; i < s.H; ++i) t[i] = (cnt[order[i]] + own_slots + 1) / 2;
   return t;
-}
-
-// Pieces of a head under a longest run of `lmax` tiles (0: the whole head).
-inline int pieces_for(int tiles, int lmax) { return lmax > 0 ? (tiles + lmax - 1) / lmax : 1; }
-// Every piece of an equal cut must hold at least one tile.
-inline bool cut_ok(int tiles, int ns) { return ns >= 1 && (ns - 1) * ((tiles + ns - 1) / ns) < tiles; }
-
-SplitShape shape_of(const std::vector<int>& tiles, const std::vector<int>& ns, int n_qp) {
-  SplitShape r;
-  for (size_t i = 0; i < tiles.size(); ++i) {
-    r.items += n_qp * ns[i];
-    if (ns[i] > 1) { r.slots += n_qp * ns[i]; r.ctrs += n_qp; }
-  }
-  return r;
-}
-
-// Estimated makespan (in units of one 128-key tile) of the launch.  Items are taken by the resident CTAs in
-// dispatch order (heads by descending key count, pieces, query tile pairs, sequences interleaved); for very
-// large launches the list-scheduling bound total / SMs + longest is used.  The per-item constants were fitted
-// to clock stamps of the kernel: an item costs its tiles plus the result's way out and the next item's start;
-// a piece writes fp32 partials instead, and the piece that arrives last reads the others.
-double makespan_of(const std::vector<int>& tiles, const std::vector<int>& ns, int n_qp, int n_seq, int n_sm) {
-  constexpr double FIXED = 2.0, PUBLISH = 1.0, MERGE_PER_PIECE = 1.5;
-  std::vector<double> costs;
-  double total = 0.0, longest = 0.0;
-  for (size_t i = 0; i < tiles.size(); ++i) {
-    const int piece = (tiles[i] + ns[i] - 1) / ns[i];
-    for (int pc = 0; pc < ns[i]; ++pc) {
-      const int len = std::min(tiles[i], (pc + 1) * piece) - pc * piece;
-      const double c = len + FIXED + (ns[i] > 1 ? PUBLISH + MERGE_PER_PIECE * (ns[i] - 1) / ns[i] : 0.0);
-      for (int q = 0; q < n_qp; ++q) costs.push_back(c);
-      total += c * n_qp;
-      longest = std::max(longest, c);
-    }
-  }
-  const size_t n_items = costs.size() * (size_t)n_seq;
-  if (n_items > 8192) return total * n_seq / n_sm + longest;
-  std::vector<double> sm(n_sm, 0.0);                       // binary min-heap of SM finish times
-  auto cmp = [](double a, double b) { return a > b; };
-  for (double c : costs)
-    for (int q = 0; q < n_seq; ++q) {
-      std::pop_heap(sm.begin(), sm.end(), cmp);
-      sm.back() += c;
-      std::push_heap(sm.begin(), sm.end(), cmp);
-    }
-  return *std::max_element(sm.begin(), sm.end());
 }
 
 // Head table of a call whose sequences all follow one schedule (generic kernel): heads in dispatch order with
@@ -335,7 +277,6 @@ void fill_head_table(heatkv_ctx* ctx, const int* seq_ids, int n_seq, int step, i
 // cut further so that the last round of items fills the SMs.  It is cached per (schedule, step, layer, batch
 // size).  Calls that mix schedules use one longest run for all of them.
 void choose_split(heatkv_ctx* ctx, const int* seq_ids, int n_seq, int step, int layer, AttnParams* p) {
-  constexpr int MIN_PIECE = 4;                              // shorter pieces measured slower (their fixed cost dominates)
   const int n_qp = (p->t_q + 255) / 256, own_slots = (p->n_own + HEATKV_PAGE_TOKENS - 1) / HEATKV_PAGE_TOKENS;
   const PlanEntry& pe0 = *ctx->plans[ctx->seqs[seq_ids[0]].plan];
   bool one_plan = pe0.sched.H <= 64;
@@ -346,43 +287,15 @@ void choose_split(heatkv_ctx* ctx, const int* seq_ids, int n_seq, int step, int 
   const uint64_t key = (pe0.uid << 24) ^ ((uint64_t)step << 20) ^ ((uint64_t)layer << 8) ^ (uint64_t)n_seq ^
                        (one_plan ? 0ull : 1ull << 63);
   auto fits = [&](const SplitShape& sh) {
-    return (uint64_t)sh.slots * n_seq <= ctx->split_slots && (uint64_t)sh.ctrs * n_seq * 8 <= ctx->split_ctrs;
+    return (uint64_t)sh.slots * n_seq <= ctx->split_slots &&
+           (uint64_t)sh.ctrs * n_seq * SPLIT_CTRS_PER_GROUP <= ctx->split_ctrs;
   };
   auto it = ctx->split_choice.find(key);
-  if (it == ctx->split_choice.end()) {
-    SplitChoice best;
-    best.ns.assign(H, 1);
-    double best_t = makespan_of(tiles, best.ns, n_qp, n_seq, ctx->n_sm);
-    const int max_tiles = *std::max_element(tiles.begin(), tiles.end());
-    std::vector<int> lmaxes = {0};
-    for (int div : {2, 3, 4, 6, 8, 12, 16}) {
-      const int cand = (max_tiles + div - 1) / div;
-      if (cand < MIN_PIECE) break;
-      lmaxes.push_back(cand);
-    }
-    for (int lmax : lmaxes) {
-      std::vector<int> base(H);
-      for (int i = 0; i < H; ++i) base[i] = pieces_for(tiles[i], lmax);
-      // heads dispatched last (the shortest) cut into `extra` times as many pieces; only with a per-head table
-      for (int extra = 1; extra <= (one_plan ? 3 : 1); ++extra)
-        for (int tail = (extra == 1 ? 0 : 1); tail <= (extra == 1 ? 0 : H); ++tail) {
-          std::vector<int> ns = base;
-          bool ok = true;
-          for (int i = H - tail; i < H; ++i) {
-            ns[i] = base[i] * extra;
-            ok = ok && cut_ok(tiles[i], ns[i]) && (tiles[i] + ns[i] - 1) / ns[i] >= MIN_PIECE;
-          }
-          for (int i = 0; i < H; ++i) ok = ok && cut_ok(tiles[i], ns[i]);
-          if (!ok || (lmax == 0 && tail == 0)) continue;
-          if (!fits(shape_of(tiles, ns, n_qp))) continue;
-          const double t = makespan_of(tiles, ns, n_qp, n_seq, ctx->n_sm);
-          if (t < 0.95 * best_t) { best_t = t; best.ns = ns; best.lmax = tail == 0 ? lmax : -1; }
-        }
-    }
-    it = ctx->split_choice.emplace(key, std::move(best)).first;
-  }
+  if (it == ctx->split_choice.end())
+    it = ctx->split_choice.emplace(key, split_search(tiles, n_qp, n_seq, ctx->n_sm, one_plan, ctx->split_slots,
+                                                     ctx->split_ctrs)).first;
   const SplitChoice& ch = it->second;
-  SplitShape m = shape_of(tiles, ch.ns, n_qp);
+  SplitShape m = split_shape(tiles, ch.ns, n_qp);
   int lmax = ch.lmax > 0 ? ch.lmax : 0;
   if (!one_plan) {
     // other schedules in the batch follow the same longest run; the per-sequence bounds cover all of them
@@ -395,8 +308,8 @@ void choose_split(heatkv_ctx* ctx, const int* seq_ids, int n_seq, int step, int 
         last_plan = pi;
         const std::vector<int> t = ordered_tiles(*ctx->plans[pi], step, layer, own_slots);
         std::vector<int> ns(t.size());
-        for (size_t k = 0; k < t.size(); ++k) ns[k] = pieces_for(t[k], lm);
-        const SplitShape sh = shape_of(t, ns, n_qp);
+        for (size_t k = 0; k < t.size(); ++k) ns[k] = split_pieces_for(t[k], lm);
+        const SplitShape sh = split_shape(t, ns, n_qp);
         b.items = std::max(b.items, sh.items); b.slots = std::max(b.slots, sh.slots); b.ctrs = std::max(b.ctrs, sh.ctrs);
       }
       return b;

@@ -69,6 +69,28 @@ struct Plan {
   const PlanHeader& header() const { return *reinterpret_cast<const PlanHeader*>(blob.data()); }
 };
 
+// ---- key-range splitting of the tensor-memory attention launch (split.cpp)
+constexpr int SPLIT_MIN_PIECE = 4;        // shorter pieces measured slower (their fixed cost dominates)
+constexpr int SPLIT_CTRS_PER_GROUP = 8;   // arrival counters per (head, query tile pair): one per 32 rows
+// How one attention launch cuts its heads: pieces per head in dispatch order; `lmax` > 0 when that is the
+// same as "no run longer than lmax tiles" (the rule a call with several schedules applies to all of them).
+struct SplitChoice {
+  std::vector<int> ns;
+  int lmax = 0;
+};
+// Items of one sequence: count, partial slots, counter groups.
+struct SplitShape {
+  int items = 0, slots = 0, ctrs = 0;
+};
+// Pieces of a head under a longest run of `lmax` tiles (0: the whole head).
+inline int split_pieces_for(int tiles, int lmax) { return lmax > 0 ? (tiles + lmax - 1) / lmax : 1; }
+// Every piece of an equal cut must hold at least one tile.
+inline bool split_cut_ok(int tiles, int ns) { return ns >= 1 && (ns - 1) * ((tiles + ns - 1) / ns) < tiles; }
+SplitShape split_shape(const std::vector<int>& tiles, const std::vector<int>& ns, int n_qp);
+double split_makespan(const std::vector<int>& tiles, const std::vector<int>& ns, int n_qp, int n_seq, int n_sm);
+SplitChoice split_search(const std::vector<int>& tiles, int n_qp, int n_seq, int n_sm, bool per_head, uint64_t max_slots,
+                         uint64_t max_ctrs);
+
 int build_schedule(const heatkv_config& cfg, const double* scas, const double* cas, int policy,
                    int accounting, double b, const double* fraction, Schedule* out);
 int build_plan(const Schedule& sch, int layout, Plan* out);

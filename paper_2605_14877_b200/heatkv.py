@@ -21,7 +21,7 @@ __all__ = [
     "heatkv_create", "heatkv_destroy", "heatkv_calibrate_scores", "heatkv_calibrate_scores_static",
     "heatkv_finalize_scores", "heatkv_build_schedule", "heatkv_schedule_free", "heatkv_schedule_masks", "heatkv_schedule_footprint",
     "heatkv_schedule_plan", "heatkv_seq_open", "heatkv_seq_close", "heatkv_append_compact", "heatkv_scale_attention",
-    "heatkv_attention_append",
+    "heatkv_attention_append", "heatkv_split_plan",
     "heatkv_cache_bytes", "heatkv_retained_indices", "heatkv_export_head", "heatkv_allocator_stats",
     "heatkv_launch_count", "heatkv_device_status", "heatkv_strerror", "heatkv_attention_split", "arena_bytes_for",
 ]
@@ -92,7 +92,7 @@ def exported_symbols():
             "heatkv_build_schedule", "heatkv_schedule_free", "heatkv_schedule_masks",
             "heatkv_schedule_footprint", "heatkv_schedule_plan", "heatkv_seq_open", "heatkv_seq_close", "heatkv_append_compact",
             "heatkv_scale_attention", "heatkv_attention_append", "heatkv_cache_bytes", "heatkv_retained_indices", "heatkv_export_head",
-            "heatkv_attention_split", "heatkv_allocator_stats", "heatkv_launch_count", "heatkv_device_status",
+            "heatkv_attention_split", "heatkv_split_plan", "heatkv_allocator_stats", "heatkv_launch_count", "heatkv_device_status",
             "heatkv_strerror"]
 
 
@@ -125,6 +125,8 @@ _lib.heatkv_scale_attention.argtypes = [_P, C.POINTER(C.c_int), C.c_int, C.c_int
                                         C.POINTER(Strides), _P, _P, _P]
 _lib.heatkv_attention_append.argtypes = [_P, C.POINTER(C.c_int), C.c_int, C.c_int, C.c_int, _P, _P, _P,
                                          C.POINTER(Strides), _P, _P, _P]
+_lib.heatkv_split_plan.argtypes = [C.POINTER(C.c_int32), C.c_int, C.c_int, C.c_int, C.c_int, C.c_int, C.c_uint64, C.c_uint64,
+                                   C.POINTER(C.c_int32), C.POINTER(C.c_double), C.POINTER(C.c_double)]
 _lib.heatkv_attention_split.argtypes = [_P, C.POINTER(C.c_int), C.c_int, C.c_int, C.c_int, C.POINTER(C.c_int32),
                                         C.POINTER(C.c_int32)]
 _lib.heatkv_cache_bytes.argtypes = [_P, C.c_int, C.POINTER(C.c_uint64), C.POINTER(C.c_uint64)]
@@ -282,11 +284,24 @@ def heatkv_attention_append(ctx, seq_ids, layer, step, q, k_new, v_new, strides,
 
 
 def heatkv_attention_split(ctx, seq_ids, layer, step):
-    """(longest run of 128-key tiles per CTA, 0 = whole heads; CTAs of the launch) for this attention call."""
+    """(longest piece in 128-key tiles among the heads that are cut, 0 = whole heads; work items of the launch)
+    for this attention call."""
     ids, n = _ids(seq_ids)
     a, b = C.c_int32(), C.c_int32()
     _check(_lib.heatkv_attention_split(ctx, ids, n, layer, step, C.byref(a), C.byref(b)), "heatkv_attention_split")
     return a.value, b.value
+
+
+def heatkv_split_plan(tiles, n_qp: int, n_seq: int, n_sm: int = 148, per_head: bool = True,
+                      max_slots: int = 1 << 40, max_ctrs: int = 1 << 40):
+    """Pieces per head (tiles in descending order) and the estimated makespans (whole heads, chosen cut)."""
+    n = len(tiles)
+    t = (C.c_int32 * n)(*[int(x) for x in tiles])
+    out = (C.c_int32 * n)()
+    a, b = C.c_double(), C.c_double()
+    _check(_lib.heatkv_split_plan(t, n, n_qp, n_seq, n_sm, int(per_head), max_slots, max_ctrs, out, C.byref(a), C.byref(b)),
+           "heatkv_split_plan")
+    return [int(x) for x in out], a.value, b.value
 
 
 def heatkv_cache_bytes(ctx: int, seq_id: int):

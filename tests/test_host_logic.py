@@ -287,3 +287,61 @@ def test_scas_rank_dispersion_matches_oracle():
     runs = rng.random((7, 3, 4, 9))
     runs[2, 1, 2, 5] = runs[2, 0, 1, 5]                        # a tie: broken by head index on both sides
     assert np.allclose(scas_rank_dispersion(runs, 3), O.scas_rank_dispersion(runs, 3), rtol=0, atol=1e-12)
+
+
+# ---- key-range splitting of the attention launch (pure host search, no GPU)
+def _pieces_valid(tiles, pieces, min_piece=4):
+    for t, n in zip(tiles, pieces):
+        assert n >= 1
+        piece = -(-t // n)
+        assert (n - 1) * piece < t                      # every piece holds at least one tile
+        if n > 1:
+            assert piece >= min_piece
+
+
+def test_split_plan_leaves_full_launches_whole():
+    import paper_2605_14877_b200 as hk
+    # 64 (sequence, head) units x 16 query tile pairs of equal length: 1024 items for 148 SMs, nothing to gain
+    pieces, whole, cut = hk.heatkv_split_plan([34] * 32, n_qp=16, n_seq=2)
+    assert pieces == [1] * 32 and cut == whole
+
+
+def test_split_plan_cuts_few_long_heads():
+    import paper_2605_14877_b200 as hk
+    # 2 heads, one query tile pair, 83 key tiles each: two items for 148 SMs
+    pieces, whole, cut = hk.heatkv_split_plan([83, 83], n_qp=1, n_seq=1)
+    _pieces_valid([83, 83], pieces)
+    assert min(pieces) > 1 and cut < 0.95 * whole
+    # the scratch region bounds the cut: no slots, no cut
+    pieces0, _, _ = hk.heatkv_split_plan([83, 83], n_qp=1, n_seq=1, max_slots=0)
+    assert pieces0 == [1, 1]
+    # a longest-run rule (calls that mix schedules): equal heads get equal piece counts
+    pieces1, _, _ = hk.heatkv_split_plan([83, 83], n_qp=1, n_seq=1, per_head=False)
+    assert pieces1[0] == pieces1[1] > 1
+
+
+def test_split_plan_ragged_heads_and_invariants():
+    import paper_2605_14877_b200 as hk
+    rng = np.random.default_rng(0)
+    for _ in range(40):
+        H = int(rng.integers(1, 40))
+        tiles = sorted((int(x) for x in rng.integers(1, 90, size=H)), reverse=True)
+        n_qp, n_seq = int(rng.integers(1, 17)), int(rng.integers(1, 9))
+        pieces, whole, cut = hk.heatkv_split_plan(tiles, n_qp=n_qp, n_seq=n_seq)
+        _pieces_valid(tiles, pieces)
+        assert cut <= whole                              # a cut is only taken when the estimate improves
+        if pieces != [1] * H:
+            assert cut < 0.95 * whole
+    # one long head among a few short ones that cannot fill the SMs: the long head is cut, the short ones are not
+    tiles = [60] + [8] * 5
+    pieces, whole, cut = hk.heatkv_split_plan(tiles, n_qp=2, n_seq=2)
+    _pieces_valid(tiles, pieces)
+    assert pieces[0] >= 2 and cut < whole and all(n <= 2 for n in pieces[1:])
+
+
+def test_split_plan_rejects_bad_input():
+    import paper_2605_14877_b200 as hk
+    with pytest.raises(hk.HeatKVError):
+        hk.heatkv_split_plan([3, 5], n_qp=1, n_seq=1)       # not in dispatch (descending) order
+    with pytest.raises(hk.HeatKVError):
+        hk.heatkv_split_plan([4, 0], n_qp=1, n_seq=1)
