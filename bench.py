@@ -600,17 +600,20 @@ def main():
     beta = torch.zeros(shape.L, shape.H, shape.K, shape.K, dtype=torch.float32, device=dev)
     ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     calib_ms = 0.0
-    for seed in CALIB_SEEDS:
+    for i, seed in enumerate([CALIB_SEEDS[0]] + list(CALIB_SEEDS)):
+        # the first pass is a warm-up into a scratch accumulator (first launches load the kernels), not timed
+        acc = torch.zeros_like(beta) if i == 0 else beta
         q, k, v = W.qkv_layer(shape, seed, 0, device=dev)
         ev0.record()
         for step in range(shape.K):
             lo, hi = ses.step_slices(step)
             qs, ks = q[:, :, lo:hi], k[:, :, :hi]
             hk.heatkv_calibrate_scores(ses.ctx, 0, step, n_seq, qs, ks, None, hk.Strides.of(qs, ks), bias[0, step],
-                                       beta, None)
+                                       acc, None)
         ev1.record()
         torch.cuda.synchronize()
-        calib_ms += ev0.elapsed_time(ev1)
+        if i > 0:
+            calib_ms += ev0.elapsed_time(ev1)
         del q, k, v
     _, scas, _ = hk.heatkv_finalize_scores(ses.ctx, beta, len(CALIB_SEEDS) * n_seq, shape.L, shape.H, shape.K)
     sch = ses.schedule(scas=scas, b=B_BUDGET)
