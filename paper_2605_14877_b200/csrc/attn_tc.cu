@@ -720,18 +720,19 @@ attn_tc_kernel(const __grid_constant__ AttnParams p, const __grid_constant__ Map
             last = __shfl_sync(0xffffffffu, last, 0);
             if (last) {
               __threadfence();
-              float m_all = m_ref;                                    // common reference and total row sum
+              // The pieces are added in piece order, this warp's own (still in TMEM) at its place among them, so
+              // the result does not depend on which piece happened to arrive last.
+              float m_all = -INFINITY;                                // common reference and total row sum
               for (int s2 = 0; s2 < n_split; ++s2) {
-                if (s2 == piece) continue;
                 const float* sl = slots + (int64_t)(s2 * n_qp + qp) * SPLIT_SLOT_FLOATS;
-                m_all = fmaxf(m_all, __ldcg(sl + 2 * BM * D + x * BM + row));
+                m_all = fmaxf(m_all, s2 == piece ? m_ref : __ldcg(sl + 2 * BM * D + x * BM + row));
               }
-              const float w_own = exp2f(m_ref - m_all);
-              float l_all = l_sum * w_own;
+              float l_all = 0.f;
               for (int s2 = 0; s2 < n_split; ++s2) {
-                if (s2 == piece) continue;
                 const float* sl = slots + (int64_t)(s2 * n_qp + qp) * SPLIT_SLOT_FLOATS;
-                l_all += __ldcg(sl + 2 * BM * D + 2 * BM + x * BM + row) * exp2f(__ldcg(sl + 2 * BM * D + x * BM + row) - m_all);
+                const float l2 = s2 == piece ? l_sum : __ldcg(sl + 2 * BM * D + 2 * BM + x * BM + row);
+                const float m2 = s2 == piece ? m_ref : __ldcg(sl + 2 * BM * D + x * BM + row);
+                l_all = fmaf(l2, exp2f(m2 - m_all), l_all);
               }
               const float inv = 1.f / l_all;
 #pragma unroll 1
@@ -741,9 +742,14 @@ attn_tc_kernel(const __grid_constant__ AttnParams p, const __grid_constant__ Map
                 tmem_wait_ld();
                 float acc[32];
 #pragma unroll
-                for (int i = 0; i < 32; ++i) acc[i] = __uint_as_float(r[i]) * w_own;
+                for (int i = 0; i < 32; ++i) acc[i] = 0.f;
                 for (int s2 = 0; s2 < n_split; ++s2) {
-                  if (s2 == piece) continue;
+                  if (s2 == piece) {
+                    const float w_own = exp2f(m_ref - m_all);
+#pragma unroll
+                    for (int i = 0; i < 32; ++i) acc[i] = fmaf(__uint_as_float(r[i]), w_own, acc[i]);
+                    continue;
+                  }
                   const float* sl = slots + (int64_t)(s2 * n_qp + qp) * SPLIT_SLOT_FLOATS;
                   const float w = exp2f(__ldcg(sl + 2 * BM * D + x * BM + row) - m_all);
                   const float4* oc = reinterpret_cast<const float4*>(sl) + (c * 8) * (2 * BM) + x * BM + row;

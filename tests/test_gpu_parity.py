@@ -258,6 +258,30 @@ def test_key_range_splitting_is_used_and_exact(hk):
                      kernel=hk.KERNEL_AUTO)
 
 
+def test_split_heads_are_reproducible_bit_for_bit(hk):
+    """Pieces of a cut head are merged in piece order whichever arrives last: the same generation run four
+    times gives identical output bits (steps of this workload are cut, see the test above)."""
+    from paper_2605_14877_b200.sweep import Session
+    sh = W.Shape("split", L=1, H=3, d=128, sides=W.SIDES_13[:12], n_seq=2, s=3)
+    scores = W.synthetic_scas(sh, 3)
+    q, k, v = W.qkv_layer(sh, 0, 0, device="cuda")
+    runs = []
+    with Session(sh.L, sh.H, sh.d, sh.t, sh.s, pool_rows=sh.n_seq * sh.H * (sh.c[-2] + 64 * sh.K)) as ses:
+        sch = ses.schedule(scas=scores, b=0.6)
+        for _ in range(4):
+            ids = [hk.heatkv_seq_open(ses.ctx, sch) for _ in range(sh.n_seq)]
+            out = torch.zeros_like(q)
+            ses.generate(ids, lambda l: (q, k, v), lambda l: out, fused=True)
+            torch.cuda.synchronize()
+            runs.append(W.bf16_bits(out).copy())
+            for i in ids:
+                hk.heatkv_seq_close(ses.ctx, i)
+        assert hk.heatkv_device_status(ses.ctx) == 0
+        hk.heatkv_schedule_free(sch)
+    for r in runs[1:]:
+        assert np.array_equal(r, runs[0])
+
+
 def test_full_budget_equals_uncompressed(hk):
     sh = W.Shape("full", L=1, H=2, d=64, sides=W.SIDES_13[:9], n_seq=1, s=2)
     scores = W.synthetic_scas(sh, 1)
