@@ -136,6 +136,21 @@ def attention_flops(shape, am, n_seq):
     return out
 
 
+def attention_bytes(shape, am, n_seq):
+    """Algorithmic bytes of every (step) attention launch: K and V of the visible keys plus Q and O, bf16,
+    summed over (seq, head): 2*2*d*n_vis + 2*2*d*t_k."""
+    t = shape.t
+    out = []
+    for k in range(shape.K):
+        tot = 0
+        for l in range(shape.L):
+            for h in range(shape.H):
+                prior = sum(t[i] for i in range(k) if (int(am[k, l, h]) >> i) & 1)
+                tot += 4 * shape.d * (prior + t[k]) + 4 * shape.d * t[k]
+        out.append(tot * n_seq)
+    return out
+
+
 def oracle_context(shape):
     """Inputs of the oracle timing: the oracle's own schedule from seeded scores, one sequence of
     the workload widened to fp64."""
@@ -619,6 +634,7 @@ def main():
     sch = ses.schedule(scas=scas, b=B_BUDGET)
     am, km, nk, budget = hk.heatkv_schedule_masks(sch, shape.K, shape.L, shape.H)
     flops = attention_flops(shape, am, n_seq)
+    by = attention_bytes(shape, am, n_seq)
     calib_flops = sum(2 * shape.d * shape.t[k] * shape.c[k] for k in range(shape.K)) * shape.H * n_seq * len(CALIB_SEEDS)
     tc_steps = [kk for kk in range(shape.K) if args.kernel != "generic" and (shape.t[kk] >= 256 or args.kernel == "tcgen05")]
 
@@ -795,6 +811,7 @@ def main():
         "work_items_per_scale": [int(c[1]) for c in cuts],
         "longest_piece_tiles_per_scale": [int(c[0]) for c in cuts],
         "attention_tflops_per_scale": [round(flops[kk] / (float(attn_ms[kk]) * 1e-3) / 1e12, 1) for kk in range(shape.K)],
+        "attention_algorithmic_gb_per_s_per_scale": [round(by[kk] / (float(attn_ms[kk]) * 1e-3) / 1e9, 1) for kk in range(shape.K)],
         "attention_tflops_all_scales": sum(flops) / (float(attn_ms.sum()) * 1e-3) / 1e12,
         "images_per_s_32_layers_extrapolated": value / 32.0,
         "calibration": {"ms_per_sample_batch": calib_ms / len(CALIB_SEEDS),
