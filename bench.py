@@ -40,7 +40,7 @@ METRIC = "images_per_sec_scale_step_attention_2b_single_layer_20x"
 UNIT = "images/s"
 # dram__bytes_read.sum + dram__bytes_write.sum of the dominant kernel's launches of one sweep, from the ncu
 # capture summarised under profiles/; None once the kernel changed after the capture
-TRAFFIC_BYTES_PER_SWEEP = 318.9e6
+TRAFFIC_BYTES_PER_SWEEP = 314.8e6
 
 
 def peaks():
