@@ -3,23 +3,24 @@
 // The launch is a list of work items handed out through a counter: one CTA per SM stays resident and takes
 // item after item, so the loads and first products of the next item run under the epilogue of the current
 // one.  An attention item is 256 queries of one (sequence, head) as two 128-row tiles A and B that share
-// the key/value stream, over the head's whole key range or one piece of it; the items after them store
-// the step's own K/V (when the call carries the cache update).  Warp roles:
+// the key/value stream, over the head's whole key range or one piece of it.  When the call carries the
+// cache update, the rows of the step's own K/V are copied by two otherwise idle warps, which take
+// destination half-tiles from a counter of their own.  Warp roles:
 //   warp 0      fetches and decodes items (a two-entry ring in shared memory) and is the TMA producer:
 //               Q tiles once per item, then K and V half-tiles (64 rows x 128 dims each) gathered
 //               through the plan's page table, followed by the step's own keys.
 //   warp 1      MMA issuer: S = Q K^T and O += P V with tcgen05.mma, accumulators in TMEM.
+//   warps 2-3   cache update (only when the call carries it).
 //   warps 4-7   softmax of tile A, warps 8-11 softmax of tile B: one thread per query row
 //               reads its row of S from TMEM, keeps the running max / sum, writes P (bf16)
 //               back into the columns S occupied, and rescales O only when the row max grew
 //               by more than 2^8 since the last reference (the sum keeps the same reference,
-//               so the result is exact).  The same warps write the item's result and copy the
-//               rows of a cache-update item.
+//               so the result is exact).  The same warps write the item's result.
 // TMEM columns: S_A/P_A 0..127, S_B/P_B 128..255, O_A 256..383, O_B 384..511.
 // The MMA order S_A S_B (PV_A S_A' PV_B S_B')* lets the softmax of one tile overlap the
-// tensor work of the other.  Heads whose key range is longer than the launch's limit are cut into pieces
-// whose unnormalised results meet in a scratch region, where, for every group of 32 rows, the warp that
-// arrives last merges them.  All barrier phases run on across items.  Every wait is bounded; on expiry the
+// tensor work of the other.  The host may cut a head's key range into pieces (a count per head); their
+// unnormalised results meet in a scratch region, where, for every group of 32 rows, the warp that arrives
+// last adds them up in piece order.  All barrier phases run on across items.  Every wait is bounded; on expiry the
 // CTA records a status word, drains its own copies and leaves.
 #include <algorithm>
 
