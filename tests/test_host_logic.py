@@ -107,6 +107,27 @@ def test_schedule_ties_break_by_head_index(hk):
     assert np.array_equal(am, ram) and np.array_equal(km, rkm)
 
 
+def test_schedule_matches_hand_worked_pop_order(hk):
+    """The C++ builder against the hand-derived GreedyEarlyPruning instance (Sec. 3.3, Algorithm 1: Sort of
+    R_k by layer descending, source scale descending, rank ascending) -- expected values come from the
+    golden file, not from the oracle."""
+    from golden_reader import read_early_pruning_instance
+    inst, cases = read_early_pruning_instance()
+    L, H, K = inst["L"], inst["H"], len(inst["sides"])
+    t = [a * a for a in inst["sides"]]
+    cfg = hk.Config.make(L, H, 64, t, inst["s"])
+    for case in cases:
+        accs = {"physical": [0], "printed": [1], "both": [0, 1]}[case["accounting"]]
+        for acc in accs:
+            sch = hk.heatkv_build_schedule(cfg, scas=inst["scas_array"], cas=inst["cas_array"],
+                                           policy=1 if case["policy"] == "binary" else 0, accounting=acc, b=inst["b"])
+            am, _, nk, B = hk.heatkv_schedule_masks(sch, K, L, H)
+            hk.heatkv_schedule_free(sch)
+            assert B == inst["B"] and list(nk[:-1]) == inst["N"]
+            for (k, layer, head), vis in case["visible"].items():
+                assert am[k - 1, layer - 1, head - 1] == sum(1 << (i - 1) for i in vis), (case["policy"], acc, k, layer, head)
+
+
 def test_explicit_policy_matches_oracle(hk):
     sh = W.TINY
     frac = np.array([W.TINY_FRACTIONS])

@@ -357,6 +357,40 @@ def _greedy_vs_brute_force(seed):
 
 
 # ------------------------------------------------------------------ cache contents + bytes (P8, P9)
+def _golden_early_pruning_cases():
+    from golden_reader import read_early_pruning_instance
+    inst, cases = read_early_pruning_instance()
+    out = []
+    for case in cases:
+        accs = {"physical": [O.ACCOUNT_PHYSICAL], "printed": [O.ACCOUNT_LITERAL],
+                "both": [O.ACCOUNT_PHYSICAL, O.ACCOUNT_LITERAL]}[case["accounting"]]
+        for acc in accs:
+            out.append((inst, case, acc))
+    return out
+
+
+@pytest.mark.parametrize("inst,case,accounting", _golden_early_pruning_cases(),
+                         ids=lambda x: x["policy"] if isinstance(x, dict) and "policy" in x else None)
+def test_early_pruning_pop_order_hand_worked(inst, case, accounting):
+    """Sec. 3.3 / Algorithm 1, the Sort of R_k: candidates leave by layer descending, then source scale
+    descending (head-scale policy), then rank ascending.  The expected E_k and visible sets come from a
+    derivation written out by hand in tests/golden/early_pruning_order.txt; with either secondary key
+    reversed the instance yields a different E_4."""
+    binary = case["policy"] == "binary"
+    scores = inst["cas_array"] if binary else inst["scas_array"]
+    sch = O.heatkv_schedule(scores, inst["b"], inst["s"], inst["sides"],
+                            O.POLICY_BINARY if binary else O.POLICY_HEATKV, accounting)
+    assert sch.B == inst["B"] and list(sch.N) == inst["N"]
+    K = sch.K
+    for k, want in case["E"].items():
+        got = {(i + 1, l + 1, h + 1) for i in range(K) for l in range(sch.L) for h in range(sch.H) if sch.E[k - 1][i, l, h]}
+        if binary:   # the file lists heads; a popped head takes all its non-sink source scales with it
+            want = {(i, l, h) for (l, h) in want for i in range(inst["s"] + 1, K)}
+        assert got == want, (k, got, want)
+    for (k, layer, head), vis in case["visible"].items():
+        assert O.visible_scales(sch, k, layer - 1, head - 1) == vis, (k, layer, head)
+
+
 def test_cache_contents_brute_force_and_bytes():
     sh = W.Shape("small", L=3, H=4, d=64, sides=W.SIDES_13[:8], n_seq=1, s=2)
     scores = W.synthetic_scas(sh, 2)
