@@ -1,12 +1,12 @@
 #!/usr/bin/env python
 """Benchmark of the HeatKV hot path on B200.
 
-One "step" = one whole generation sweep of the 2B-class single-layer workload (16 heads,
-d=128, 13 scales = 10 521 tokens, batch 2 = one cond/uncond image pair, 20x KV compression):
-for every scale, the eviction before the scale, the ragged attention over the retained keys
-plus the scale's own keys, and the append/compaction of the new K/V.  The schedule comes
-from the library's own calibration kernel run once on seeded samples before timing (the
-paper computes it offline, once per model and budget).
+One "step" = one image (a cond/uncond pair, batch 2) through the attention + cache path of a 2B-class model:
+32 layers of the single-layer workload (16 heads, d=128, 13 scales = 10 521 tokens, 20x KV compression), every
+layer with seeded activations of its own.  A layer's sweep is, for every scale, the eviction before the scale,
+the ragged attention over the retained keys plus the scale's own keys, and the append/compaction of the new
+K/V.  The schedule comes from the library's own calibration kernel run once on seeded samples before timing
+(the paper computes it offline, once per model and budget).  MLP, VAE and text encoder are not part of it.
 
     python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference]
 
@@ -36,11 +36,39 @@ import heatkv_workloads as W  # noqa: E402
 B_BUDGET = 1.0 / 20.0
 CALIB_SEEDS = (100, 101, 102, 103)
 DATA_SEED = 0
-METRIC = "images_per_sec_scale_step_attention_2b_single_layer_20x"
+METRIC = "images_per_sec_scale_step_attention_2b_class_20x"
+N_LAYERS = 32            # layers of the 2B-class model: one step replays the layer sweep this many times
 UNIT = "images/s"
-# dram__bytes_read.sum + dram__bytes_write.sum of the dominant kernel's launches of one sweep, from the ncu
-# capture summarised under profiles/; None once the kernel changed after the capture
-TRAFFIC_BYTES_PER_SWEEP = 314.8e6
+# dram__bytes_read.sum + dram__bytes_write.sum of the dominant kernel's seven launches of one layer sweep, from
+# the ncu capture summarised in profiles/attn_tc_kernel_config2.md, with the sources the captured kernel was
+# built from (first 16 hex digits of their SHA-256); reported as null once either file has changed
+TRAFFIC_CAPTURE = {"bytes_per_layer_sweep": 314.8e6,
+                   "sources": {"attn_tc.cu": "3c8ec421b8bcdbb8", "tc_common.cuh": "4dbc238674fe2b73"}}
+
+
+def captured_traffic():
+    import hashlib
+    for name, want in TRAFFIC_CAPTURE["sources"].items():
+        path = os.path.join(ROOT, "paper_2605_14877_b200", "csrc", name)
+        try:
+            got = hashlib.sha256(open(path, "rb").read()).hexdigest()[:16]
+        except OSError:
+            return None
+        if got != want:
+            return None
+    return TRAFFIC_CAPTURE["bytes_per_layer_sweep"]
+
+
+def oracle_threads():
+    """Threads the oracle's numpy really computes with: those of the BLAS behind its matrix products."""
+    try:
+        import threadpoolctl
+        n = [int(x["num_threads"]) for x in threadpoolctl.threadpool_info() if x.get("user_api") == "blas"]
+        if n:
+            return max(n)
+    except Exception:
+        pass
+    return 1
 
 
 def peaks():
@@ -190,10 +218,10 @@ def oracle_seconds(shape, ctx, head, steps):
 
 
 def oracle_images_per_s(shape, ctx, samples):
-    """samples: list of (head, steps).  Extrapolates to one image (n_seq * H units, all scales) by
-    algorithmic flops.  Returns (images/s, seconds spent, flops covered / flops of one image)."""
+    """samples: list of (head, steps).  Extrapolates to one image (N_LAYERS layers of n_seq * H units, all scales)
+    by algorithmic flops.  Returns (images/s, seconds spent, flops covered / flops of one image)."""
     all_steps = list(range(1, shape.K + 1))
-    image_flops = shape.n_seq * sum(oracle_flops(shape, ctx, h, all_steps) for h in range(shape.H))
+    image_flops = N_LAYERS * shape.n_seq * sum(oracle_flops(shape, ctx, h, all_steps) for h in range(shape.H))
     secs = sum(oracle_seconds(shape, ctx, h, st) for h, st in samples)
     done = sum(oracle_flops(shape, ctx, h, st) for h, st in samples)
     return done / secs / image_flops, secs, done / image_flops
@@ -215,29 +243,28 @@ def run_reference(args, rank):
     stride = max(1, int(math.ceil(args.steps * unit_s / budget_s)))
     samples = [(i % shape.H, [st for st in all_steps if (st + i) % stride == 0] or [shape.K]) for i in range(args.steps)]
     value, secs, frac = oracle_images_per_s(shape, ctx, samples)
-    threads = torch.get_num_threads()
-    sample = (f"per step one (seq, head) unit of {shape.n_seq * shape.H}, every {stride}-th scale "
+    threads = oracle_threads()
+    sample = (f"per step one (layer, seq, head) unit of {N_LAYERS * shape.n_seq * shape.H}, every {stride}-th scale "
               f"(all 13 when 1); {secs:.1f} s of CPU work = {frac:.3g} images, extrapolated by flops")
     line = {"impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus,
             "steps": args.steps, "warmup": args.warmup, "ms_per_step": 1e3 / value,
             "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
             "config": {"workload": shape.name, "L": shape.L, "H": shape.H, "d": shape.d, "scales": shape.K,
                        "tokens": shape.n_tokens, "n_seq": shape.n_seq, "budget": B_BUDGET, "policy": "heatkv",
-                       "s": shape.s},
+                       "s": shape.s, "layers": N_LAYERS},
             "cpu_baseline": {"value": value, "unit": UNIT, "cores": threads, "kind": "oracle", "sample": sample},
             "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
             "gpu_launches": 0}
     print(json.dumps(line), flush=True)
 
 
-def run_cache_workload(args):
-    """Cache-update kernels at a saturating shape (not the headline line): the larger-model layer shape
-    (32 heads, d=128, 16 sequences, one layer).  Appends are timed with every head storing (full
-    budget, paged and ragged); the in-place compaction of the ragged layout under a 1/5 budget.
-    Bytes are algorithmic: 8*d*t_k per storing head (K and V, read + write), 8*d*moved tokens per move."""
+def cache_update_numbers(reps, cases=("append_paged", "append_ragged", "compact_ragged"), first_scale=1):
+    """Cache-update kernels at a saturating shape: the larger-model layer shape (32 heads, d=128, 16 sequences,
+    one layer).  Appends are timed with every head storing (full budget, paged and ragged); the in-place
+    compaction of the ragged layout under a 1/5 budget.  Bytes are algorithmic: 8*d*t_k per storing head (K and
+    V, read + write), 8*d*moved tokens per move.  Rows for scales >= first_scale."""
     import paper_2605_14877_b200 as hk
     from paper_2605_14877_b200.sweep import Session
-    torch.cuda.set_device(0)
     sh = W.Shape("larger_layer", L=1, H=32, d=128, sides=W.SIDES_13, n_seq=16, s=3)
     pk = peaks()
     out = {"workload": "cache_update_saturating", "shape": {"H": sh.H, "d": sh.d, "n_seq": sh.n_seq, "scales": sh.K},
@@ -248,12 +275,13 @@ def run_cache_workload(args):
     stream = torch.cuda.current_stream()
     for name, layout, b in (("append_paged", hk.LAYOUT_PAGED, 1.0), ("append_ragged", hk.LAYOUT_RAGGED, 1.0),
                             ("compact_ragged", hk.LAYOUT_RAGGED, 0.2)):
+        if name not in cases:
+            continue
         ses = Session(sh.L, sh.H, sh.d, sh.t, sh.s, pool_rows=sh.n_seq * sh.H * (sh.c[-2] + 64 * sh.K) + 64, layout=layout)
         sch = ses.schedule(scas=W.synthetic_scas(sh, 0), b=b)
         am, km, nk, _ = hk.heatkv_schedule_masks(sch, sh.K, sh.L, sh.H)
         plan = hk.heatkv_schedule_plan(sch, layout)
         ms = np.zeros(sh.K)
-        reps = max(3, min(args.steps, 10))
         for rep in range(reps + 1):
             ids = [hk.heatkv_seq_open(ses.ctx, sch) for _ in range(sh.n_seq)]
             for step in range(sh.K - 1):
@@ -275,7 +303,7 @@ def run_cache_workload(args):
                 hk.heatkv_seq_close(ses.ctx, i)
         rows = []
         hdr = plan[:20]
-        for step in range(sh.K - 1):
+        for step in range(first_scale - 1, sh.K - 1):
             storing = sum(1 for h in range(sh.H) if (int(km[step, 0, h]) >> step) & 1)
             nbytes = 8 * sh.d * sh.t[step] * storing * sh.n_seq
             if name == "compact_ragged":
@@ -295,9 +323,18 @@ def run_cache_workload(args):
                              "GBs": round(nbytes / (ms[step] * 1e-3) / 1e9, 1),
                              "frac": round(nbytes / (ms[step] * 1e-3) / 1e9 / pk["hbm_gbs"], 3)})
         out[name] = rows
+        st = hk.heatkv_kernel_launches(ses.ctx)
+        out[name + "_kernels"] = {"append_kernel": int(st.append), "compact_kernel": int(st.compact)}
         hk.heatkv_schedule_free(sch)
         ses.close()
-    print(json.dumps(out), flush=True)
+    del ks, vs, flush
+    torch.cuda.empty_cache()
+    return out
+
+
+def run_cache_workload(args):
+    torch.cuda.set_device(0)
+    print(json.dumps(cache_update_numbers(max(3, min(args.steps, 10)))), flush=True)
 
 
 def run_few_heads_workload(args):
@@ -544,13 +581,13 @@ def run_model_workload(args, which):
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=300)
+    ap.add_argument("--steps", type=int, default=50)
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--layout", default="paged", choices=["paged", "ragged"])
     ap.add_argument("--kernel", default="auto", choices=["auto", "generic", "tcgen05"])
     ap.add_argument("--launch", default="graph", choices=["graph", "eager"],
-                    help="timed sweeps replay one captured CUDA graph of the 13-step sweep, or issue every call")
+                    help="timed steps replay one captured CUDA graph of the 32 x 13 launches, or issue every call")
     ap.add_argument("--calls", default="fused", choices=["fused", "separate"],
                     help="fused: heatkv_attention_append (one launch per step in the paged layout); separate: "
                          "heatkv_scale_attention followed by heatkv_append_compact")
@@ -638,18 +675,23 @@ def main():
     calib_flops = sum(2 * shape.d * shape.t[k] * shape.c[k] for k in range(shape.K)) * shape.H * n_seq * len(CALIB_SEEDS)
     tc_steps = [kk for kk in range(shape.K) if args.kernel != "generic" and (shape.t[kk] >= 256 or args.kernel == "tcgen05")]
 
-    # ---- device-resident inputs of the timed workload: one [n_seq, H, t_k, d] block per scale
-    q, k, v = W.qkv_layer(shape, DATA_SEED, 0, device=dev)
-    qs_, ks_, vs_, os_ = [], [], [], []
-    for step in range(shape.K):
-        lo, hi = ses.step_slices(step)
-        qs_.append(q[:, :, lo:hi].contiguous()); ks_.append(k[:, :, lo:hi].contiguous())
-        vs_.append(v[:, :, lo:hi].contiguous()); os_.append(torch.zeros_like(qs_[-1]))
-    del q, k, v
+    # ---- device-resident inputs of the timed workload: per layer, one [n_seq, H, t_k, d] block per scale
+    # (N_LAYERS x 345 MB: every layer reads activations of its own, far more than the L2 holds)
+    layer_bufs = []
+    for layer in range(N_LAYERS):
+        q, k, v = W.qkv_layer(shape, DATA_SEED, layer, device=dev)
+        bq, bk, bv, bo = [], [], [], []
+        for step in range(shape.K):
+            lo, hi = ses.step_slices(step)
+            bq.append(q[:, :, lo:hi].contiguous()); bk.append(k[:, :, lo:hi].contiguous())
+            bv.append(v[:, :, lo:hi].contiguous()); bo.append(torch.zeros_like(bq[-1]))
+        layer_bufs.append((bq, bk, bv, bo))
+        del q, k, v
+    qs_, ks_, vs_, os_ = layer_bufs[0]
     flush = torch.empty(256 << 20, dtype=torch.uint8, device=dev)
 
     def sweep(events=None, bufs=None):
-        """One image pair through the layer: 13 x (pre-step eviction, attention, append/compaction)."""
+        """One image pair through one layer: 13 x (pre-step eviction, attention, append/compaction)."""
         stream = torch.cuda.current_stream()
         bq, bk, bv, bo = bufs or (qs_, ks_, vs_, os_)
         ids = [hk.heatkv_seq_open(ses.ctx, sch) for _ in range(n_seq)]
@@ -668,6 +710,12 @@ def main():
         for i in ids:
             hk.heatkv_seq_close(ses.ctx, i)
 
+    def image():
+        """One step: the image pair through all N_LAYERS layers (the context is one layer wide, so every layer
+        is a fresh pair of sequences on the same pool rows, with that layer's activations)."""
+        for layer in range(N_LAYERS):
+            sweep(bufs=layer_bufs[layer])
+
     def barrier():
         torch.cuda.synchronize()
         if dist is not None:
@@ -675,11 +723,14 @@ def main():
             torch.cuda.synchronize()
 
     for _ in range(args.warmup):
-        sweep()
+        image()
     barrier()
-    launches0 = hk.heatkv_launch_count(ses.ctx)
-    sweep()
-    launches_per_sweep = hk.heatkv_launch_count(ses.ctx) - launches0
+    launches0, kern0 = hk.heatkv_launch_count(ses.ctx), hk.heatkv_kernel_launches(ses.ctx)
+    image()
+    launches_per_step = hk.heatkv_launch_count(ses.ctx) - launches0
+    kern1 = hk.heatkv_kernel_launches(ses.ctx)
+    per_step_kernels = {n: int(getattr(kern1, n) - getattr(kern0, n)) for n in
+                        ("attention_tcgen05", "attention_generic", "append", "compact")}
     graph = None
     if args.launch == "graph":
         # the calls are plain launches on the current stream once the schedule's plan is resident, so the
@@ -687,17 +738,17 @@ def main():
         side = torch.cuda.Stream()
         side.wait_stream(torch.cuda.current_stream())
         with torch.cuda.stream(side):
-            sweep()
+            image()
         torch.cuda.current_stream().wait_stream(side)
         barrier()
         graph = torch.cuda.CUDAGraph()
         with torch.cuda.graph(graph):
-            sweep()
+            image()
         for _ in range(args.warmup):
             graph.replay()
         barrier()
 
-    # ---- timed region: exactly K sweeps, L2 flushed (untimed) before each
+    # ---- timed region: exactly K steps (images), L2 flushed (untimed) before each
     stream = torch.cuda.current_stream()
     sampler = ClockSampler(local)
     sampler.start()
@@ -710,17 +761,18 @@ def main():
         if graph is not None:
             graph.replay()
         else:
-            sweep()
+            image()
         step_events[it][1].record(stream)
     barrier()
     total_ms = sum(a.elapsed_time(b) for a, b in step_events)
 
-    # ---- kernel durations: the same K sweeps issued call by call with events around every attention launch
+    # ---- kernel durations: layer sweeps issued call by call with events around every attention launch
+    n_kern = max(N_LAYERS, min(args.steps, 64))
     kern_events = [{kk: (torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True))
-                    for kk in range(shape.K)} for _ in range(args.steps)]
-    for it in range(args.steps):
+                    for kk in range(shape.K)} for _ in range(n_kern)]
+    for it in range(n_kern):
         flush.fill_(it & 0xff)
-        sweep(kern_events[it])
+        sweep(kern_events[it], layer_bufs[it % N_LAYERS])
     barrier()
     clocks = sampler.stop()
     per_step_ms = np.array([[ke[kk][0].elapsed_time(ke[kk][1]) for kk in range(shape.K)] for ke in kern_events])
@@ -731,11 +783,12 @@ def main():
     for i in ids_:
         hk.heatkv_seq_close(ses.ctx, i)
 
-    # ---- end to end: the same sweep from pinned host buffers, copies inside the timed region
-    h2d = 3 * sum(x.numel() for x in qs_) * 2
-    d2h = sum(x.numel() for x in qs_) * 2
+    # ---- end to end: the same step from pinned host buffers, copies inside the timed region.  Every layer's
+    # Q/K/V go up and its output comes down (one pinned set serves all layers: the bytes moved are what counts).
+    h2d = N_LAYERS * 3 * sum(x.numel() for x in qs_) * 2
+    d2h = N_LAYERS * sum(x.numel() for x in qs_) * 2
     e2e_ms = float("nan")
-    e2e_steps = max(3, min(args.steps, 20))
+    e2e_steps = max(3, min(args.steps, 5))
     if not args.no_e2e:
         hq, hkk, hv = ([x.cpu().pin_memory() for x in xs] for xs in (qs_, ks_, vs_))
         hout = [torch.empty_like(x).pin_memory() for x in hq]
@@ -780,7 +833,8 @@ def main():
         e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
         e0.record(stream)
         for _ in range(e2e_steps):
-            sweep_e2e()
+            for _layer in range(N_LAYERS):
+                sweep_e2e()
         e1.record(stream)
         barrier()
         e2e_ms = max(e0.elapsed_time(e1), 1e3 * (time.perf_counter() - t0)) / e2e_steps
@@ -788,7 +842,21 @@ def main():
     # ---- aggregate over ranks (replicas): slowest rank's time
     ms_per_step, value, e2e_value = aggregate_replicas(total_ms, e2e_ms, args.steps, dist, dev)   # one image pair per replica
 
-    # ---- roofline of the dominant kernel: attn_tc_kernel (tcgen05), all its launches of a sweep
+    # ---- which kernels ran (the library's own count), and the cache-update kernels at their saturating shape
+    ks1 = hk.heatkv_kernel_launches(ses.ctx)
+    if args.kernel != "generic":
+        assert ks1.tcgen05_attention_ready == 1 and per_step_kernels["attention_tcgen05"] == N_LAYERS * len(tc_steps), per_step_kernels
+    dominant = ("tc::attn_tc_kernel<%d> (tcgen05.mma, TMEM accumulators, TMA gathers)" % shape.d
+                if per_step_kernels["attention_tcgen05"] else "attn_generic_kernel<%d> (mma.sync)" % shape.d)
+    cache_update = None
+    if rank == 0 and world == 1 and args.layout == "paged":
+        cu = cache_update_numbers(5, cases=("append_paged", "compact_ragged"), first_scale=9)
+        cache_update = {"shape": cu["shape"], "peak_gbs": cu["peak_gbs"], "peak_source": cu["peak_source"],
+                        "append_kernel_paged": cu["append_paged"], "append_plus_compact_kernel_ragged_budget_1_5": cu["compact_ragged"],
+                        "kernels_launched": {"append_paged": cu["append_paged_kernels"], "compact_ragged": cu["compact_ragged_kernels"]},
+                        "bytes": "algorithmic: 8*d*t_k per storing head, 8*d per moved token"}
+
+    # ---- roofline of the dominant kernel, all its launches of a layer sweep
     pk = peaks()
     attn_ms = per_step_ms.mean(axis=0)                            # [K] mean duration per launch
     dom_flops = sum(flops[kk] for kk in tc_steps)
@@ -803,9 +871,13 @@ def main():
         "config": {"workload": shape.name, "L": shape.L, "H": shape.H, "d": shape.d, "scales": shape.K,
                    "tokens": shape.n_tokens, "n_seq": n_seq, "budget": B_BUDGET, "policy": "heatkv", "s": shape.s,
                    "layout": args.layout, "kernel": args.kernel, "launch": args.launch, "calls": args.calls,
-                   "l2": "256 MB flush write between timed steps",
-                   "one_image": "cond/uncond pair through one layer; x32 layers for a 2B-class model",
+                   "layers": N_LAYERS,
+                   "l2": "256 MB flush write between timed steps; every layer reads its own 345 MB of activations",
+                   "one_image": "cond/uncond pair through the attention + cache path of 32 layers (the single-layer "
+                                "workload replayed per layer with that layer's seeded activations); MLP/VAE/text not included",
                    "n_k": [int(x) for x in nk], "replicas": world},
+        "ms_per_layer_sweep": ms_per_step / N_LAYERS,
+        "image_pairs_per_s_one_layer": value * N_LAYERS,
         "effective_kv_tb_per_s": uncompressed_kv_bytes / (float(attn_ms.sum()) * 1e-3) / 1e12,
         "attention_ms_per_scale": [round(float(x), 5) for x in attn_ms],
         "work_items_per_scale": [int(c[1]) for c in cuts],
@@ -813,28 +885,32 @@ def main():
         "attention_tflops_per_scale": [round(flops[kk] / (float(attn_ms[kk]) * 1e-3) / 1e12, 1) for kk in range(shape.K)],
         "attention_algorithmic_gb_per_s_per_scale": [round(by[kk] / (float(attn_ms[kk]) * 1e-3) / 1e9, 1) for kk in range(shape.K)],
         "attention_tflops_all_scales": sum(flops) / (float(attn_ms.sum()) * 1e-3) / 1e12,
-        "images_per_s_32_layers_extrapolated": value / 32.0,
         "calibration": {"ms_per_sample_batch": calib_ms / len(CALIB_SEEDS),
                         "tflops": calib_flops / (calib_ms * 1e-3) / 1e12, "samples": len(CALIB_SEEDS) * n_seq},
-        "roofline": {"bound": "tensor", "kernel": f"attn_tc_kernel, its {len(tc_steps)} launches per sweep (scales with t_k >= 256)",
+        "kernels_per_step": per_step_kernels,
+        "roofline": {"bound": "tensor", "kernel": f"{dominant}: its {len(tc_steps)} launches per layer sweep (scales with t_k >= 256), "
+                                                  f"{per_step_kernels['attention_tcgen05']} per step",
+                     "timing": "CUDA events around each launch, call by call, mean over layer sweeps",
                      "achieved": achieved, "peak": pk["bf16_tflops"], "unit": "TFLOP/s",
                      "frac": achieved / pk["bf16_tflops"], "peak_source": pk["source"] + " burst bf16",
                      "largest_launch": {"scale": big + 1, "tflops": flops[big] / (float(attn_ms[big]) * 1e-3) / 1e12,
                                         "frac": flops[big] / (float(attn_ms[big]) * 1e-3) / 1e12 / pk["bf16_tflops"]},
-                     "traffic": TRAFFIC_BYTES_PER_SWEEP},
+                     "traffic": captured_traffic(), "traffic_unit": "bytes per layer sweep (7 launches), ncu dram read + write"},
         "e2e": {"value": e2e_value, "unit": UNIT, "h2d_bytes_per_step": h2d,
                 "d2h_bytes_per_step": d2h, "steps": e2e_steps},
-        "gpu_launches": int(launches_per_sweep * args.steps),
+        "gpu_launches": int(launches_per_step * args.steps),
         "clocks": clocks,
     }
     if rank == 0 and world == 1 and not args.no_cpu_baseline:
         ctx = oracle_context(shape)
         samples = [(h, list(range(1, shape.K + 1))) for h in (0, 3, 5, 7, 8, 11, 13, 15)] * 5
         v, secs, frac = oracle_images_per_s(shape, ctx, samples)
-        line["cpu_baseline"] = {"value": v, "unit": UNIT, "cores": torch.get_num_threads(), "kind": "oracle",
-                                "sample": f"{len(samples)} (seq, head) units of {shape.n_seq * shape.H}, all 13 scales "
+        line["cpu_baseline"] = {"value": v, "unit": UNIT, "cores": oracle_threads(), "kind": "oracle",
+                                "sample": f"{len(samples)} (layer, seq, head) units of {N_LAYERS * shape.n_seq * shape.H}, all 13 scales "
                                           f"(attention + cache contents); {secs:.1f} s of CPU work = {frac:.3g} images, "
                                           "extrapolated by flops"}
+    if cache_update is not None:
+        line["cache_update"] = cache_update
     hk.heatkv_schedule_free(sch)
     ses.close()
     if dist is not None:

@@ -99,6 +99,17 @@ typedef struct {                 /* element strides of the [n_seq, H, t, d] acti
   int64_t o_seq, o_head, o_tok;
 } heatkv_strides;
 
+typedef struct {                 /* which kernels a context has launched so far             */
+  uint32_t tcgen05_attention_ready;    /* 1: the tensor-memory attention kernel is set up on this device */
+  uint32_t tcgen05_calibration_ready;  /* 1: the tensor-memory calibration kernel is set up               */
+  uint64_t attention_tcgen05;    /* launches of the tcgen05 / TMEM / TMA attention kernel (carries the cache
+                                    update of heatkv_attention_append in the paged layout)               */
+  uint64_t attention_generic;    /* launches of the warp-level attention kernel                          */
+  uint64_t calibration_tcgen05, calibration_generic;
+  uint64_t append, compact;      /* stand-alone cache-update kernels                                     */
+  uint64_t other;                /* small helper kernels (fixed-order reduction of the static-scratch call) */
+} heatkv_kernel_stats;
+
 typedef struct {
   uint64_t pool_rows;            /* rows (tokens) the K pool and the V pool can hold        */
   uint64_t reserved_rows;        /* rows reserved by open sequences                         */
@@ -110,7 +121,11 @@ typedef struct {
 } heatkv_alloc_stats;
 
 /* Context: validates the shape, splits the arena into a metadata region and the K / V
- * pools, zero-fills the pools (enqueued on `stream`).  The arena must outlive the context. */
+ * pools, zero-fills the pools (enqueued on `stream`).  The arena must outlive the context.
+ * With kernel = HEATKV_KERNEL_AUTO or HEATKV_KERNEL_TCGEN05 the tensor-memory kernels are set up here; if that
+ * fails on a device of compute capability 10.x (or on any device under HEATKV_KERNEL_TCGEN05) the call returns
+ * HEATKV_ERR_CUDA: a context never falls back to the warp-level kernel behind the caller's back.  Which kernel
+ * ran is reported by heatkv_kernel_launches. */
 int heatkv_create(const heatkv_config* cfg /*HOST*/, void* stream, heatkv_ctx** out /*HOST*/);
 int heatkv_destroy(heatkv_ctx* ctx);
 
@@ -124,7 +139,8 @@ int heatkv_destroy(heatkv_ctx* ctx);
  *   v_full  DEVICE bf16 like k_full, or NULL when `out` is NULL
  *   seg_bias DEVICE fp32 [H][K] additive logit bias per source scale, or NULL
  *   beta_accum DEVICE fp32 [L][H][K][K], zero-initialised by the caller before the first call
- *   out     DEVICE bf16 [n_seq,H,t[step],d] strides o_*: the attention output, or NULL    */
+ *   out     DEVICE bf16 [n_seq,H,t[step],d] strides o_*: the attention output, or NULL
+ * Without an output the o_* strides are not read (they may be left zero).                */
 int heatkv_calibrate_scores(heatkv_ctx* ctx, int layer, int step, int n_seq, const void* q,
                             const void* k_full, const void* v_full, const heatkv_strides* st,
                             const float* seg_bias, float* beta_accum, void* out, void* stream);
@@ -143,7 +159,8 @@ int heatkv_calibrate_scores(heatkv_ctx* ctx, int layer, int step, int n_seq, con
  *   All calls share the one array and it keeps the last call's contents: every slot a call reads is
  *   written by that call first, so nothing needs clearing, but two calls whose kernels overlap on the
  *   GPU (different streams) race on it -- keep them on one stream or order them yourself.
- * Arguments as in heatkv_calibrate_scores.  Results agree with it up to the order of the fp32 sums. */
+ * Arguments as in heatkv_calibrate_scores (the o_* strides are not read).  Results agree with it up to the
+ * order of the fp32 sums. */
 int heatkv_calibrate_scores_static(heatkv_ctx* ctx, int layer, int step, int n_seq, const void* q,
                                    const void* k_full, const heatkv_strides* st, const float* seg_bias,
                                    float* beta_accum, void* stream);
@@ -203,10 +220,10 @@ int heatkv_seq_close(heatkv_ctx* ctx, int seq_id);
 /* Sec. 3.3 -- cache update for one layer.
  *   k_new != NULL: after layer `layer` ran at `step`: store the step's K/V for every head
  *     whose (step,l,h) is not in G_step and drop the head-scales of G_step \ A_step of this
- *     layer ("evicted immediately after their layer has executed").  The last step stores
+ *     layer (Sec. 3.3: these leave right after their own layer has run).  The last step stores
  *     nothing.  k_new, v_new DEVICE bf16 [n_seq,H,t[step],d], strides kv_*.
- *   k_new == NULL: before `step` starts: drop the head-scales of E_step ("evicted before
- *     scale k starts") in `layer`, or in all layers when layer < 0.
+ *   k_new == NULL: before `step` starts: drop the head-scales of E_step (Sec. 3.3, Algorithm 1:
+ *     the early-pruned set, gone before the scale begins) in `layer`, or in all layers when layer < 0.
  * Survivors keep their order.  In the paged layout eviction moves no data.               */
 int heatkv_append_compact(heatkv_ctx* ctx, const int* seq_ids /*HOST*/, int n_seq, int layer,
                           int step, const void* k_new, const void* v_new,
@@ -225,7 +242,7 @@ int heatkv_scale_attention(heatkv_ctx* ctx, const int* seq_ids /*HOST*/, int n_s
                            void* stream);
 
 /* heatkv_scale_attention followed by heatkv_append_compact(k_new != NULL) for the same (layer, step), as one
- * call: the order a model issues them in (Sec. 3.3: evictions "immediately after their layer has executed").
+ * call: the order a model issues them in (Sec. 3.3: G_step \ A_step is evicted as soon as its layer has run).
  * In the paged layout both run in ONE kernel launch (the plan releases the pages of G_step \ A_step only
  * after the layer's append, so the new scale never lands on a page this step's attention still reads): on
  * the tensor-memory kernel two spare warps per SM copy the new rows beside the attention work, whatever the
@@ -260,7 +277,13 @@ int heatkv_split_plan(const int32_t* tiles /*HOST*/, int n_heads, int n_qp, int 
                       double* makespan_cut);
 
 /* Introspection (host state only unless noted). */
-int heatkv_cache_bytes(heatkv_ctx* ctx, int seq_id, uint64_t* actual, uint64_t* reserved);
+/* Bytes of K and V the sequence holds right now, two ways: *actual = the pool rows its plan has placed for the
+ * head-scales it stores (valid rows of their destination half-tiles) x d x 2 (K and V) x 2 bytes; *closed_form =
+ * sum over (layer, head) of kept_tokens x d x 2 x 2 from the schedule's masks (Sec. 3.2: the cache size in
+ * tokens).  The two agree unless the plan and the schedule have come apart.  Either may be NULL. */
+int heatkv_cache_bytes(heatkv_ctx* ctx, int seq_id, uint64_t* actual, uint64_t* closed_form);
+/* The pool rows reserved for the sequence: first row and row count (x d x 2 x 2 bytes of K and V). */
+int heatkv_seq_reservation(heatkv_ctx* ctx, int seq_id, uint64_t* first_row, uint64_t* rows);
 /* Global token indices c_{i-1}+j of the tokens head (layer, head) holds now; idx HOST with
  * room for c_{K-1} entries. */
 int heatkv_retained_indices(heatkv_ctx* ctx, int seq_id, int layer, int head, int32_t* idx, int* n);
@@ -271,6 +294,15 @@ int heatkv_export_head(heatkv_ctx* ctx, int seq_id, int layer, int head, void* k
 int heatkv_allocator_stats(heatkv_ctx* ctx, heatkv_alloc_stats* out);
 /* Kernels launched by this context so far. */
 int heatkv_launch_count(heatkv_ctx* ctx, uint64_t* n);
+/* The same per kernel, with the state of the tensor-memory kernels' set-up. */
+int heatkv_kernel_launches(heatkv_ctx* ctx, heatkv_kernel_stats* out);
+/* Appendix on S-CAS stability -- how much the head ordering moves between calibration sets.  scas_runs HOST
+ * [n_runs][L][H][K]: S-CAS of n_runs independent calibration sets (heatkv_finalize_scores).  For every prunable
+ * source scale k (s <= k <= K-2, 0-based) each run ranks the L*H heads by ascending S-CAS (ties by ascending
+ * l*H+h, as heatkv_build_schedule does); out[k] = mean over heads of the standard deviation (population form)
+ * of the head's rank position over the runs; 0 for the other k.  out HOST [K].  Pure host code.
+ * HEATKV_ERR_NAN_SCORE if a score is not finite. */
+int heatkv_rank_dispersion(const double* scas_runs, int n_runs, int L, int H, int K, int s, double* out);
 /* Reads the device-side status word (synchronises `stream`): HEATKV_OK or
  * HEATKV_ERR_DEVICE_TIMEOUT if a bounded wait inside a kernel ran out. */
 int heatkv_device_status(heatkv_ctx* ctx, void* stream);

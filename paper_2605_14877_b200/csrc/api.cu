@@ -19,6 +19,7 @@ cudaError_t launch_compact(const CopyParams& p, int n_seq, cudaStream_t stream);
 struct TcState;
 int tc_create(const heatkv_config& cfg, void* k_pool, void* v_pool, uint64_t pool_rows, TcState** out);
 void tc_destroy(TcState* st);
+bool tc_ready(const TcState* st);
 bool tc_supported(const TcState* st, const AttnParams& p, int d, int n_seq, bool calib);
 cudaError_t launch_attn_tc(TcState* st, const AttnParams& p, int d, int n_seq, bool calib, cudaStream_t stream,
                            int* launches);
@@ -27,6 +28,7 @@ struct CalibTcState;
 uint64_t calib_tc_desc_bytes(const heatkv_config& cfg);
 int calib_tc_create(const heatkv_config& cfg, void* dev_table, cudaStream_t stream, CalibTcState** out);
 void calib_tc_destroy(CalibTcState* st);
+bool calib_tc_ready(const CalibTcState* st);
 bool calib_tc_supported(const CalibTcState* st, const AttnParams& p, int d, int n_seq);
 cudaError_t launch_calib_tc(CalibTcState* st, const AttnParams& p, int n_seq, cudaStream_t stream);
 }  // namespace heatkv
@@ -114,6 +116,7 @@ struct heatkv_ctx {
   std::vector<Seq> seqs;
   uint64_t reserved_rows = 0, peak_reserved = 0, meta_used = 0;
   uint64_t launches = 0;
+  heatkv_kernel_stats kstats = {};             // launches per kernel
   TcState* tc = nullptr;
   CalibTcState* calib_tc = nullptr;
   // key-range splitting of the tensor-memory attention kernel
@@ -193,7 +196,7 @@ bool pre_needed(const Schedule& s, int step, int l) {
   return false;
 }
 
-int check_strides(const heatkv_ctx* ctx, const heatkv_strides* st, int t, heatkv_strides* out) {
+int check_strides(const heatkv_ctx* ctx, const heatkv_strides* st, int t, heatkv_strides* out, bool has_output = true) {
   const int64_t d = ctx->cfg.d, H = ctx->cfg.H;
   if (!st) {
     out->q_tok = out->kv_tok = out->o_tok = d;
@@ -202,6 +205,9 @@ int check_strides(const heatkv_ctx* ctx, const heatkv_strides* st, int t, heatkv
     return HEATKV_OK;
   }
   *out = *st;
+  if (!has_output) {                               // nothing is written: the caller may leave o_* unset
+    out->o_seq = out->q_seq; out->o_head = out->q_head; out->o_tok = out->q_tok;
+  }
   const int64_t* v = &out->q_seq;
   for (int i = 0; i < 9; ++i)
     if (v[i] < 0 || (v[i] & 7)) return HEATKV_ERR_INVALID_ARG;
@@ -420,7 +426,10 @@ int heatkv_create(const heatkv_config* cfg, void* stream_, heatkv_ctx** out) {
   if (cudaMemsetAsync(ctx->meta, 0, STATUS_BYTES, stream) != cudaSuccess) return HEATKV_ERR_CUDA;
   if (cudaMemsetAsync(ctx->k_pool, 0, 2 * rows * row_bytes, stream) != cudaSuccess) return HEATKV_ERR_CUDA;
   int rc = tc_create(ctx->cfg, ctx->k_pool, ctx->v_pool, rows, &ctx->tc);
-  if (rc != HEATKV_OK) return rc;
+  if (rc != HEATKV_OK) {
+    tc_destroy(ctx->tc);
+    return rc;
+  }
   // the calibration kernel's half-tile table (key rows cut at source-scale borders) sits in the metadata region
   void* calib_table = nullptr;
   {
@@ -431,6 +440,16 @@ int heatkv_create(const heatkv_config* cfg, void* stream_, heatkv_ctx** out) {
     }
   }
   rc = calib_tc_create(ctx->cfg, calib_table, stream, &ctx->calib_tc);
+  // A context that may use the tensor-memory kernels must really have them: on a device of compute capability
+  // 10.x a failed set-up (driver entry point, tensor maps, shared-memory or register limits) is an error, never
+  // a quiet switch to the warp-level kernel.  HEATKV_KERNEL_TCGEN05 demands them on any device.
+  if (rc == HEATKV_OK && cfg->kernel != HEATKV_KERNEL_GENERIC) {
+    int dev = 0, major = 0;
+    const bool sm100 = cudaGetDevice(&dev) == cudaSuccess &&
+                       cudaDeviceGetAttribute(&major, cudaDevAttrComputeCapabilityMajor, dev) == cudaSuccess && major == 10;
+    const bool have = tc_ready(ctx->tc) && (calib_tc_ready(ctx->calib_tc) || !calib_table);
+    if (!have && (sm100 || cfg->kernel == HEATKV_KERNEL_TCGEN05)) rc = HEATKV_ERR_CUDA;
+  }
   if (rc != HEATKV_OK) {
     tc_destroy(ctx->tc);
     calib_tc_destroy(ctx->calib_tc);
@@ -610,10 +629,12 @@ static int attention_impl(heatkv_ctx* ctx, const int* seq_ids, int n_seq, int la
     }
     e = launch_attn_tc(ctx->tc, p, ctx->cfg.d, n_seq, false, stream, &n);
     ctx->launches += n;
+    ctx->kstats.attention_tcgen05 += n;
   } else {
     fill_head_table(ctx, seq_ids, n_seq, step, layer, &p);
     e = launch_attn_generic(p, ctx->cfg.d, n_seq, false, stream);
     ctx->launches += 1;
+    ctx->kstats.attention_generic += 1;
   }
   if (e != cudaSuccess) return HEATKV_ERR_CUDA;
   if (!with_update) return HEATKV_OK;
@@ -673,7 +694,7 @@ int heatkv_calibrate_scores(heatkv_ctx* ctx, int layer, int step, int n_seq, con
     s.q_head = s.o_head = d * t; s.kv_head = d * c;
     s.q_seq = s.o_seq = d * t * H; s.kv_seq = d * c * H;
   } else {
-    int rc = check_strides(ctx, st, ctx->cfg.t[step], &s);
+    int rc = check_strides(ctx, st, ctx->cfg.t[step], &s, out != nullptr);
     if (rc != HEATKV_OK) return rc;
   }
   fill_common(ctx, &p, s);
@@ -694,6 +715,7 @@ int heatkv_calibrate_scores(heatkv_ctx* ctx, int layer, int step, int n_seq, con
   cudaError_t e = use_tc ? launch_calib_tc(ctx->calib_tc, p, n_seq, stream)
                          : launch_attn_generic(p, ctx->cfg.d, n_seq, true, stream);
   ctx->launches += 1;
+  (use_tc ? ctx->kstats.calibration_tcgen05 : ctx->kstats.calibration_generic) += 1;
   return e == cudaSuccess ? HEATKV_OK : HEATKV_ERR_CUDA;
 }
 
@@ -713,7 +735,7 @@ int heatkv_calibrate_scores_static(heatkv_ctx* ctx, int layer, int step, int n_s
     s.q_head = s.o_head = d * t; s.kv_head = d * c;
     s.q_seq = s.o_seq = d * t * H; s.kv_seq = d * c * H;
   } else {
-    int rc = check_strides(ctx, st, ctx->cfg.t[step], &s);
+    int rc = check_strides(ctx, st, ctx->cfg.t[step], &s, false);
     if (rc != HEATKV_OK) return rc;
   }
   fill_common(ctx, &p, s);
@@ -730,6 +752,8 @@ int heatkv_calibrate_scores_static(heatkv_ctx* ctx, int layer, int step, int n_s
   if (too_large) return HEATKV_ERR_TOO_LARGE;
   if (e != cudaSuccess) return HEATKV_ERR_CUDA;
   ctx->launches += 2;
+  ctx->kstats.calibration_generic += 1;
+  ctx->kstats.other += 1;
   return HEATKV_OK;
 }
 
@@ -806,6 +830,7 @@ int heatkv_append_compact(heatkv_ctx* ctx, const int* seq_ids, int n_seq, int la
       p.phase = 0; p.layer_begin = l0; p.n_layers = l1 - l0; p.layer = l0;
       if (launch_compact(p, n_seq, stream) != cudaSuccess) return HEATKV_ERR_CUDA;
       ctx->launches += 1;
+      ctx->kstats.compact += 1;
     }
     for (int i = 0; i < n_seq; ++i)
       for (int l = l0; l < l1; ++l) ctx->seqs[seq_ids[i]].pre_step[l] = (int16_t)step;
@@ -817,7 +842,7 @@ int heatkv_append_compact(heatkv_ctx* ctx, const int* seq_ids, int n_seq, int la
   int rc = gather_seqs(ctx, seq_ids, n_seq, layer, step, p.seqs);
   if (rc != HEATKV_OK) return rc;
   heatkv_strides s;
-  rc = check_strides(ctx, st, ctx->cfg.t[step], &s);
+  rc = check_strides(ctx, st, ctx->cfg.t[step], &s, false);
   if (rc != HEATKV_OK) return rc;
   p.kv_seq = s.kv_seq; p.kv_head = s.kv_head; p.kv_tok = s.kv_tok;
   p.k_new = static_cast<const __nv_bfloat16*>(k_new);
@@ -831,29 +856,50 @@ int heatkv_append_compact(heatkv_ctx* ctx, const int* seq_ids, int n_seq, int la
         p.phase = 1; p.layer_begin = layer; p.n_layers = 1;
         if (launch_compact(p, n_seq, stream) != cudaSuccess) return HEATKV_ERR_CUDA;
         ctx->launches += 1;
+        ctx->kstats.compact += 1;
       }
     }
     if (launch_append(p, n_seq, stream) != cudaSuccess) return HEATKV_ERR_CUDA;
     ctx->launches += 1;
+    ctx->kstats.append += 1;
   }
   for (int i = 0; i < n_seq; ++i) ctx->seqs[seq_ids[i]].done_step[layer] = (int16_t)step;
   return HEATKV_OK;
 }
 
-int heatkv_cache_bytes(heatkv_ctx* ctx, int seq_id, uint64_t* actual, uint64_t* reserved) {
+int heatkv_cache_bytes(heatkv_ctx* ctx, int seq_id, uint64_t* actual, uint64_t* closed_form) {
   if (!ctx) return HEATKV_ERR_INVALID_ARG;
   Seq* q = get_seq(ctx, seq_id);
   if (!q) return HEATKV_ERR_INVALID_ARG;
-  const Schedule& s = ctx->plans[q->plan]->sched;
-  uint64_t tokens = 0;
+  const PlanEntry& pe = *ctx->plans[q->plan];
+  const Schedule& s = pe.sched;
+  const PlanHeader& hd = pe.plan.header();
+  const int32_t* blob = pe.plan.blob.data();
+  const Desc* descs = reinterpret_cast<const Desc*>(blob + hd.off_desc);
+  uint64_t tokens = 0, placed = 0;
   for (int l = 0; l < s.L; ++l)
     for (int h = 0; h < s.H; ++h) {
-      uint16_t m = stored_mask(ctx, *q, l, h);
-      for (int i = 0; i < s.K; ++i)
-        if ((m >> i) & 1) tokens += s.t[i];
+      const uint16_t m = stored_mask(ctx, *q, l, h);
+      for (int i = 0; i < s.K; ++i) {
+        if (!((m >> i) & 1)) continue;
+        tokens += s.t[i];
+        // rows the plan gave this head-scale when it was appended (valid rows of its destination half-tiles)
+        const size_t u = s.at(i, l, h);
+        const int32_t b0 = blob[hd.off_app_begin + u], cnt = blob[hd.off_app_cnt + u];
+        for (int j = 0; j < cnt; ++j) placed += descs[b0 + j].meta & 0xff;
+      }
     }
-  if (actual) *actual = tokens * ctx->cfg.d * 2 * 2;
-  if (reserved) *reserved = q->rows * ctx->cfg.d * 2 * 2;
+  if (actual) *actual = placed * ctx->cfg.d * 2 * 2;
+  if (closed_form) *closed_form = tokens * ctx->cfg.d * 2 * 2;
+  return HEATKV_OK;
+}
+
+int heatkv_seq_reservation(heatkv_ctx* ctx, int seq_id, uint64_t* first_row, uint64_t* rows) {
+  if (!ctx) return HEATKV_ERR_INVALID_ARG;
+  Seq* q = get_seq(ctx, seq_id);
+  if (!q) return HEATKV_ERR_INVALID_ARG;
+  if (first_row) *first_row = q->base_row;
+  if (rows) *rows = q->rows;
   return HEATKV_OK;
 }
 
@@ -930,7 +976,7 @@ int heatkv_allocator_stats(heatkv_ctx* ctx, heatkv_alloc_stats* out) {
     if (ctx->seqs[i].open) {
       out->open_seqs++;
       uint64_t bytes = 0;
-      heatkv_cache_bytes(ctx, (int)i, &bytes, nullptr);
+      heatkv_cache_bytes(ctx, (int)i, nullptr, &bytes);
       out->used_tokens += bytes / ((uint64_t)ctx->cfg.d * 4);
     }
   for (auto& pe : ctx->plans)
@@ -941,6 +987,54 @@ int heatkv_allocator_stats(heatkv_ctx* ctx, heatkv_alloc_stats* out) {
 int heatkv_launch_count(heatkv_ctx* ctx, uint64_t* n) {
   if (!ctx || !n) return HEATKV_ERR_INVALID_ARG;
   *n = ctx->launches;
+  return HEATKV_OK;
+}
+
+int heatkv_kernel_launches(heatkv_ctx* ctx, heatkv_kernel_stats* out) {
+  if (!ctx || !out) return HEATKV_ERR_INVALID_ARG;
+  *out = ctx->kstats;
+  out->tcgen05_attention_ready = tc_ready(ctx->tc) ? 1u : 0u;
+  out->tcgen05_calibration_ready = calib_tc_ready(ctx->calib_tc) ? 1u : 0u;
+  return HEATKV_OK;
+}
+
+int heatkv_rank_dispersion(const double* scas_runs, int n_runs, int L, int H, int K, int s, double* out) {
+  if (!scas_runs || !out || n_runs < 1 || L < 1 || H < 1 || K < 1 || K > HEATKV_MAX_K || s < 0 || s >= K)
+    return HEATKV_ERR_INVALID_ARG;
+  const int T = L * H;
+  try {
+    std::vector<int> order(T);
+    std::vector<double> rank((size_t)n_runs * T);
+    for (int k = 0; k < K; ++k) {
+      out[k] = 0.0;
+      if (k < s || k > K - 2) continue;                  // orders exist for the prunable source scales only
+      for (int r = 0; r < n_runs; ++r) {
+        const double* sc = scas_runs + (size_t)r * T * K;
+        for (int i = 0; i < T; ++i) {
+          if (!std::isfinite(sc[(size_t)i * K + k])) return HEATKV_ERR_NAN_SCORE;
+          order[i] = i;
+        }
+        // least to most dependent; equal scores by ascending head index, as the schedule builder orders them
+        std::stable_sort(order.begin(), order.end(),
+                         [&](int a, int b) { return sc[(size_t)a * K + k] < sc[(size_t)b * K + k]; });
+        for (int pos = 0; pos < T; ++pos) rank[(size_t)r * T + order[pos]] = (double)pos;
+      }
+      double acc = 0.0;
+      for (int i = 0; i < T; ++i) {
+        double mean = 0.0, var = 0.0;
+        for (int r = 0; r < n_runs; ++r) mean += rank[(size_t)r * T + i];
+        mean /= (double)n_runs;
+        for (int r = 0; r < n_runs; ++r) {
+          const double dlt = rank[(size_t)r * T + i] - mean;
+          var += dlt * dlt;
+        }
+        acc += std::sqrt(var / (double)n_runs);
+      }
+      out[k] = acc / (double)T;
+    }
+  } catch (const std::bad_alloc&) {
+    return HEATKV_ERR_HOST_MEMORY;
+  }
   return HEATKV_OK;
 }
 

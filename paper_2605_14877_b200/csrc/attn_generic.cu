@@ -7,6 +7,7 @@
 // from k_new.  In calibration mode (Eq. 2) every key comes from k_full and the per-row
 // probability mass of every source scale is accumulated next to the online softmax, so the
 // attention matrix alpha is never formed.
+#include <atomic>
 #include "append_device.cuh"
 
 namespace heatkv {
@@ -387,15 +388,22 @@ __global__ void reduce_partials_kernel(const float* partials, float* beta_row, i
   beta_row[(int64_t)head * K * K + sg] += acc;
 }
 
+constexpr int MAX_DEVICES = 64;
+
 template <int D, bool CALIB>
 static cudaError_t launch_one(const AttnParams& p, int n_seq, cudaStream_t stream) {
   auto kern = attn_generic_kernel<D, CALIB>;
   constexpr int bytes = CALIB ? GenericSmem<D>::BYTES : GenericSmem<D>::ATTN_BYTES;
-  static bool configured = false;
-  if (!configured) {
-    cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, bytes);
+  // the attribute belongs to the (function, device) pair: set it once on every device that launches
+  static std::atomic<bool> configured[MAX_DEVICES];
+  int dev = -1;
+  cudaError_t e = cudaGetDevice(&dev);
+  if (e != cudaSuccess) return e;
+  if (dev < 0 || dev >= MAX_DEVICES) return cudaErrorInvalidDevice;
+  if (!configured[dev].load(std::memory_order_acquire)) {
+    e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, bytes);
     if (e != cudaSuccess) return e;
-    configured = true;
+    configured[dev].store(true, std::memory_order_release);
   }
   dim3 grid((p.t_q + GM - 1) / GM + (CALIB ? 0 : p.append_tiles), CALIB ? p.H : n_seq, CALIB ? n_seq : p.H);
   kern<<<grid, GTHREADS, bytes, stream>>>(p);
@@ -413,39 +421,38 @@ cudaError_t launch_calibrate_static(const AttnParams& p_in, int d, int n_seq, cu
     *too_large = true;
     return cudaErrorInvalidValue;
   }
-  constexpr int MAX_DEVICES = 64;
-  static float* scratch_of_device[MAX_DEVICES] = {nullptr};
-  static bool configured[MAX_DEVICES][2] = {{false}};
+  static std::atomic<float*> scratch_of_device[MAX_DEVICES];
+  static std::atomic<bool> configured[MAX_DEVICES][2];
   int dev = -1;
   cudaError_t e = cudaGetDevice(&dev);
   if (e != cudaSuccess) return e;
   if (dev < 0 || dev >= MAX_DEVICES) return cudaErrorInvalidDevice;
-  if (!scratch_of_device[dev]) {
-    float* ptr = nullptr;
-    e = cudaGetSymbolAddress(reinterpret_cast<void**>(&ptr), g_static_partials);
+  float* scratch = scratch_of_device[dev].load(std::memory_order_acquire);
+  if (!scratch) {
+    e = cudaGetSymbolAddress(reinterpret_cast<void**>(&scratch), g_static_partials);
     if (e != cudaSuccess) return e;
-    scratch_of_device[dev] = ptr;
+    scratch_of_device[dev].store(scratch, std::memory_order_release);
   }
   AttnParams p = p_in;
-  p.partials = scratch_of_device[dev];
+  p.partials = scratch;
   p.out = nullptr;
   p.v_new = nullptr;
   const int which = d == 128 ? 1 : 0;
   dim3 grid(n_qtiles, p.H, n_seq);
   if (d == 128) {
     auto kern = attn_generic_kernel<128, true, true>;
-    if (!configured[dev][which]) {
+    if (!configured[dev][which].load(std::memory_order_acquire)) {
       e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, GenericSmem<128>::BYTES);
       if (e != cudaSuccess) return e;
-      configured[dev][which] = true;
+      configured[dev][which].store(true, std::memory_order_release);
     }
     kern<<<grid, GTHREADS, GenericSmem<128>::BYTES, stream>>>(p);
   } else if (d == 64) {
     auto kern = attn_generic_kernel<64, true, true>;
-    if (!configured[dev][which]) {
+    if (!configured[dev][which].load(std::memory_order_acquire)) {
       e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, GenericSmem<64>::BYTES);
       if (e != cudaSuccess) return e;
-      configured[dev][which] = true;
+      configured[dev][which].store(true, std::memory_order_release);
     }
     kern<<<grid, GTHREADS, GenericSmem<64>::BYTES, stream>>>(p);
   } else {

@@ -863,6 +863,8 @@ int tc_create(const heatkv_config& cfg, void* k_pool, void* v_pool, uint64_t poo
 
 void tc_destroy(TcState* st) { delete st; }
 
+bool tc_ready(const TcState* st) { return st && st->ready; }
+
 int tc_split_slot_floats(int d) { return d == 64 ? tc::Layout<64>::SPLIT_SLOT_FLOATS : tc::Layout<128>::SPLIT_SLOT_FLOATS; }
 
 bool tc_supported(const TcState* st, const AttnParams& p, int d, int n_seq, bool calib) {

@@ -408,6 +408,8 @@ int calib_tc_create(const heatkv_config& cfg, void* dev_table, cudaStream_t stre
 
 void calib_tc_destroy(CalibTcState* st) { delete st; }
 
+bool calib_tc_ready(const CalibTcState* st) { return st && st->ready; }
+
 bool calib_tc_supported(const CalibTcState* st, const AttnParams& p, int d, int n_seq) {
   if (!st || !st->ready || d != st->d || n_seq > 65535 || p.H > 65535) return false;
   const int64_t s[6] = {p.q_seq, p.q_head, p.q_tok, p.kv_seq, p.kv_head, p.kv_tok};

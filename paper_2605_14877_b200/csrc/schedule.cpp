@@ -2,6 +2,7 @@
 // GreedyEarlyPruning, Algorithm 2 (CacheSizeAfterLayer / CachedTokens), and the
 // per-head-fraction policy.  Everything after the sort is integer arithmetic.
 #include <algorithm>
+#include <atomic>
 #include <cmath>
 #include <numeric>
 
@@ -200,8 +201,8 @@ int build_schedule(const heatkv_config& cfg, const double* scas, const double* c
       S.keep_mask[(size_t)k * T + hd] = km;
     }
   }
-  static uint64_t next_uid = 1;
-  S.uid = next_uid++;
+  static std::atomic<uint64_t> next_uid{1};       // schedules may be built from several threads
+  S.uid = next_uid.fetch_add(1, std::memory_order_relaxed);
   *out = std::move(S);
   return HEATKV_OK;
 }

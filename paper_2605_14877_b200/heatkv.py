@@ -23,7 +23,8 @@ __all__ = [
     "heatkv_schedule_plan", "heatkv_seq_open", "heatkv_seq_close", "heatkv_append_compact", "heatkv_scale_attention",
     "heatkv_attention_append", "heatkv_split_plan",
     "heatkv_cache_bytes", "heatkv_retained_indices", "heatkv_export_head", "heatkv_allocator_stats",
-    "heatkv_launch_count", "heatkv_device_status", "heatkv_strerror", "heatkv_attention_split", "arena_bytes_for",
+    "heatkv_launch_count", "heatkv_kernel_launches", "heatkv_rank_dispersion", "heatkv_seq_reservation", "KernelStats",
+    "heatkv_device_status", "heatkv_strerror", "heatkv_attention_split", "arena_bytes_for",
 ]
 
 MAX_K, MAX_BATCH, PAGE_TOKENS = 16, 128, 64
@@ -81,6 +82,13 @@ class AllocStats(C.Structure):
                 ("open_seqs", C.c_uint32), ("plans", C.c_uint32)]
 
 
+class KernelStats(C.Structure):
+    _fields_ = [("tcgen05_attention_ready", C.c_uint32), ("tcgen05_calibration_ready", C.c_uint32),
+                ("attention_tcgen05", C.c_uint64), ("attention_generic", C.c_uint64),
+                ("calibration_tcgen05", C.c_uint64), ("calibration_generic", C.c_uint64),
+                ("append", C.c_uint64), ("compact", C.c_uint64), ("other", C.c_uint64)]
+
+
 def lib_path() -> str:
     return os.path.join(os.path.dirname(os.path.abspath(__file__)), "libheatkv.so")
 
@@ -91,9 +99,10 @@ def exported_symbols():
             "heatkv_finalize_scores",
             "heatkv_build_schedule", "heatkv_schedule_free", "heatkv_schedule_masks",
             "heatkv_schedule_footprint", "heatkv_schedule_plan", "heatkv_seq_open", "heatkv_seq_close", "heatkv_append_compact",
-            "heatkv_scale_attention", "heatkv_attention_append", "heatkv_cache_bytes", "heatkv_retained_indices", "heatkv_export_head",
-            "heatkv_attention_split", "heatkv_split_plan", "heatkv_allocator_stats", "heatkv_launch_count", "heatkv_device_status",
-            "heatkv_strerror"]
+            "heatkv_scale_attention", "heatkv_attention_append", "heatkv_cache_bytes", "heatkv_seq_reservation",
+            "heatkv_retained_indices", "heatkv_export_head",
+            "heatkv_attention_split", "heatkv_split_plan", "heatkv_allocator_stats", "heatkv_launch_count",
+            "heatkv_kernel_launches", "heatkv_rank_dispersion", "heatkv_device_status", "heatkv_strerror"]
 
 
 def _load() -> C.CDLL:
@@ -135,6 +144,9 @@ _lib.heatkv_export_head.argtypes = [_P, C.c_int, C.c_int, C.c_int, _P, _P, _P]
 _lib.heatkv_allocator_stats.argtypes = [_P, C.POINTER(AllocStats)]
 _lib.heatkv_launch_count.argtypes = [_P, C.POINTER(C.c_uint64)]
 _lib.heatkv_device_status.argtypes = [_P, _P]
+_lib.heatkv_kernel_launches.argtypes = [_P, C.POINTER(KernelStats)]
+_lib.heatkv_rank_dispersion.argtypes = [_P, C.c_int, C.c_int, C.c_int, C.c_int, C.c_int, _P]
+_lib.heatkv_seq_reservation.argtypes = [_P, C.c_int, C.POINTER(C.c_uint64), C.POINTER(C.c_uint64)]
 for _n in exported_symbols():
     if _n != "heatkv_strerror":
         getattr(_lib, _n).restype = C.c_int
@@ -305,8 +317,16 @@ def heatkv_split_plan(tiles, n_qp: int, n_seq: int, n_sm: int = 148, per_head: b
 
 
 def heatkv_cache_bytes(ctx: int, seq_id: int):
+    """(bytes of the rows the plan placed for what the sequence stores, closed form from the schedule's masks)."""
     a, r = C.c_uint64(), C.c_uint64()
     _check(_lib.heatkv_cache_bytes(ctx, seq_id, C.byref(a), C.byref(r)), "heatkv_cache_bytes")
+    return a.value, r.value
+
+
+def heatkv_seq_reservation(ctx: int, seq_id: int):
+    """(first pool row, rows) reserved for the sequence."""
+    a, r = C.c_uint64(), C.c_uint64()
+    _check(_lib.heatkv_seq_reservation(ctx, seq_id, C.byref(a), C.byref(r)), "heatkv_seq_reservation")
     return a.value, r.value
 
 
@@ -332,6 +352,21 @@ def heatkv_launch_count(ctx: int) -> int:
     n = C.c_uint64()
     _check(_lib.heatkv_launch_count(ctx, C.byref(n)), "heatkv_launch_count")
     return n.value
+
+
+def heatkv_kernel_launches(ctx: int) -> KernelStats:
+    st = KernelStats()
+    _check(_lib.heatkv_kernel_launches(ctx, C.byref(st)), "heatkv_kernel_launches")
+    return st
+
+
+def heatkv_rank_dispersion(scas_runs, s: int) -> np.ndarray:
+    """scas_runs [R, L, H, K] float64 -> [K] mean standard deviation of the heads' rank positions."""
+    a = np.ascontiguousarray(scas_runs, dtype=np.float64)
+    R, L, H, K = a.shape
+    out = np.zeros(K, dtype=np.float64)
+    _check(_lib.heatkv_rank_dispersion(_ptr(a), R, L, H, K, int(s), _ptr(out)), "heatkv_rank_dispersion")
+    return out
 
 
 def heatkv_device_status(ctx: int, stream=None) -> int:

@@ -5,7 +5,9 @@ the serving sweep (64 concurrent images, mixed per-request budgets, paged cache,
 Every (sequence, layer, head) unit runs on the GPU through the C ABI in generation order; the oracle
 checks a seeded sample of units (attention of all 13 scales within max-abs 1e-2 / mean-abs 1e-3, retained
 indices and cache contents bit-exact) and, for every unit, what holds at any size: cache bytes equal the
-closed form sum of kept tokens x d x 2 x 2 bytes, and allocator occupancy.
+closed form sum of kept tokens x d x 2 x 2 bytes, and allocator occupancy.  Besides a few fixed units the
+sample is chosen by rule (`_rule_units`): per scale from the eighth on, the heaviest and the lightest head by
+visible keys and heads long enough to be cut into pieces.
 
 Inputs: the 2B full workload uses distinct seeded Q/K/V per layer.  The two larger ones would need
 more than 160 GB of activations that way, so there all layers share one layer's seeded Q/K/V (the
@@ -43,15 +45,36 @@ def _schedule(hk, sh, scores, b):
     return sch, peak, rows
 
 
+def _rule_units(sh, ref_of, n_seq, layers, first_step=8, extra_from=7):
+    """Units picked by rule rather than by hand: for every scale from `first_step` on (the steps the tensor-memory
+    kernel cuts into pieces and dispatches by key count), the head with the most and the head with the fewest
+    visible keys among `layers`, in a sequence that rotates with the scale; every head of those layers whose key
+    range is long enough to be cut (8 key tiles of 128 and more, twice the shortest piece a cut makes) comes
+    with the heaviest.  Returned as (seq, layer, head, first step checked): these extra units are compared
+    with the oracle from scale `extra_from` on."""
+    units = {}
+    for step in range(first_step, sh.K + 1):
+        s_ = (step * 5) % n_seq
+        ref = ref_of(s_)
+        counts = {(l, h): sum(sh.t[i - 1] for i in O.visible_scales(ref, step, l, h)) + sh.t[step - 1]
+                  for l in layers for h in range(sh.H)}
+        order = sorted(counts, key=lambda lh: (counts[lh], lh))
+        picks = [order[0], order[-1]] + [lh for lh in order if counts[lh] >= 8 * 128 and lh[1] % 4 == step % 4][-2:]
+        for (l, h) in picks:
+            units.setdefault((s_, l, h), extra_from)
+    return [(s_, l, h, f) for (s_, l, h), f in sorted(units.items())]
+
+
 def _check_units(hk, ses, sh, ref, ids, units, layer_data, outs_of, bias):
-    """Oracle comparison of sampled (seq, layer, head) units after a finished generation."""
+    """Oracle comparison of sampled (seq, layer, head[, first step]) units after a finished generation."""
     sm = 1.0 / math.sqrt(sh.d)
     tot, n, worst = 0.0, 0, 0.0
-    for (s_, l, h) in units:
+    for unit in units:
+        (s_, l, h), first = unit[:3], (unit[3] if len(unit) > 3 else 1)
         q, k, v = layer_data(l)
         qh, kh, vh = _f64(q[s_, h]), _f64(k[s_, h]), _f64(v[s_, h])
         out = outs_of(l)
-        for step in range(1, sh.K + 1):
+        for step in range(first, sh.K + 1):
             lo, hi = (sh.c[step - 2] if step > 1 else 0), sh.c[step - 1]
             brow = None if bias is None else bias[l, step - 1, h].astype(np.float64)
             want = O.scale_attention(qh[lo:hi], kh, vh, ref(s_), step, l, h, sm, brow)
@@ -82,9 +105,11 @@ def test_2b_full_model_three_budgets(hk):
     bias_dev = torch.from_numpy(bias).cuda()
     layers = [W.qkv_layer(sh, 0, l, device="cuda") for l in range(sh.L)]
     outs = [torch.zeros_like(layers[l][0]) for l in range(sh.L)]
-    units = [(0, 0, 0), (3, 7, 5), (5, 18, 11), (7, 31, 15)]
+    fixed = [(0, 0, 0), (3, 7, 5), (5, 18, 11), (7, 31, 15)]
     for b in (1 / 5, 1 / 10, 1 / 20):
         ref = O.heatkv_schedule(scores, b, sh.s, sh.sides)
+        units = fixed + [u for u in _rule_units(sh, lambda s_: ref, sh.n_seq, range(sh.L)) if u[:3] not in fixed]
+        assert len(units) >= 12
         sch, peak, rows = _schedule(hk, sh, scores, b)
         assert peak <= ref.B                                      # the budget holds at every checkpoint
         with Session(sh.L, sh.H, sh.d, sh.t, sh.s, pool_rows=sh.n_seq * rows + 64, meta_bytes=64 << 20) as ses:
@@ -94,8 +119,9 @@ def test_2b_full_model_three_budgets(hk):
             assert hk.heatkv_device_status(ses.ctx) == 0
             kept = O.kept_tokens_after_step(ref, sh.K - 1)
             for i in ids:
-                actual, reserved = hk.heatkv_cache_bytes(ses.ctx, i)
-                assert actual == O.cache_bytes(kept, sh.d) and reserved >= actual
+                actual, closed = hk.heatkv_cache_bytes(ses.ctx, i)
+                reserved = hk.heatkv_seq_reservation(ses.ctx, i)[1] * sh.d * 4
+                assert actual == closed == O.cache_bytes(kept, sh.d) and reserved >= actual
             # end-of-generation size obeys the budget: N heads at c_s, the rest at c_{K-1} (Sec. 3.2)
             assert int(kept.sum()) <= ref.B
             st = hk.heatkv_allocator_stats(ses.ctx)
@@ -117,8 +143,10 @@ def test_larger_model_shape_20x(hk):
     bias_dev = torch.from_numpy(bias).cuda()
     ref = O.heatkv_schedule(scores, b, sh.s, sh.sides)
     data = W.qkv_layer(sh, 1, 0, device="cuda")
-    units = [(0, 0, 3), (9, 21, 30), (15, 39, 17)]
-    keep_layers = sorted({l for (_, l, _) in units})
+    fixed = [(0, 0, 3), (9, 21, 30), (15, 39, 17)]
+    units = fixed + [u for u in _rule_units(sh, lambda s_: ref, sh.n_seq, (0, 21, 39)) if u[:3] not in fixed]
+    assert len(units) >= 12
+    keep_layers = sorted({u[1] for u in units})
     outs = {l: torch.zeros_like(data[0]) for l in keep_layers}
     scratch_out = torch.zeros_like(data[0])
     sch, peak, rows = _schedule(hk, sh, scores, b)
@@ -129,8 +157,9 @@ def test_larger_model_shape_20x(hk):
         torch.cuda.synchronize()
         assert hk.heatkv_device_status(ses.ctx) == 0
         kept = O.kept_tokens_after_step(ref, sh.K - 1)
-        actual, reserved = hk.heatkv_cache_bytes(ses.ctx, ids[-1])
-        assert actual == O.cache_bytes(kept, sh.d)
+        actual, closed = hk.heatkv_cache_bytes(ses.ctx, ids[-1])
+        reserved = hk.heatkv_seq_reservation(ses.ctx, ids[-1])[1] * sh.d * 4
+        assert actual == closed == O.cache_bytes(kept, sh.d)
         full = sh.L * sh.H * sh.c[-2] * sh.d * 4
         assert actual <= b * full and reserved < 0.2 * full
         _check_units(hk, ses, sh, lambda s_: ref, ids, units, lambda l: data, lambda l: outs[l], bias)
@@ -151,8 +180,10 @@ def test_serving_sweep_mixed_budgets_staggered(hk):
     bias_dev = torch.from_numpy(bias).cuda()
     refs = {b: O.heatkv_schedule(scores, b, sh.s, sh.sides) for b in sorted(set(budgets))}
     data = W.qkv_layer(sh, 2, 0, device="cuda")
-    units = [(0, 0, 0), (17, 9, 4), (38, 20, 13), (63, 31, 7)]
-    keep_layers = sorted({l for (_, l, _) in units})
+    fixed = [(0, 0, 0), (17, 9, 4), (38, 20, 13), (63, 31, 7)]
+    units = fixed + [u for u in _rule_units(sh, lambda s_: refs[budgets[s_]], sh.n_seq, (0, 9, 20, 31)) if u[:3] not in fixed]
+    assert len(units) >= 12
+    keep_layers = sorted({u[1] for u in units})
     outs = {l: torch.zeros_like(data[0]) for l in keep_layers}
     scratch_out = torch.zeros_like(data[0])
     n_waves, wave = 4, sh.n_seq // 4
@@ -192,8 +223,8 @@ def test_serving_sweep_mixed_budgets_staggered(hk):
         assert st.used_tokens == want_tokens
         assert 0.3 < peak_occupancy <= 1.0, peak_occupancy
         for s_ in (0, 17, 38, 63):
-            actual, _ = hk.heatkv_cache_bytes(ses.ctx, ids[s_])
-            assert actual == O.cache_bytes(O.kept_tokens_after_step(refs[budgets[s_]], sh.K - 1), sh.d)
+            actual, closed = hk.heatkv_cache_bytes(ses.ctx, ids[s_])
+            assert actual == closed == O.cache_bytes(O.kept_tokens_after_step(refs[budgets[s_]], sh.K - 1), sh.d)
         _check_units(hk, ses, sh, lambda s_: refs[budgets[s_]], ids, units, lambda l: data, lambda l: outs[l], bias)
         for i in ids:
             hk.heatkv_seq_close(ses.ctx, i)

@@ -3,8 +3,10 @@ memory while they run (a serving loop with a memory pool fixed at start-up, a pl
 the allocator).  Its scratch is an array built into the library, so the call itself allocates nothing.
 
 The test drives the entry point through the C ABI twice in a row into one accumulator and compares it
-with two calls of heatkv_calibrate_scores on the same inputs, at the tolerance the other calibration
-tests use (1e-3 relative).  Two calls matter: the built-in array is shared by all calls and keeps the
+with two calls of heatkv_calibrate_scores on the same inputs and with the CPU oracle's beta, at the
+tolerance the other calibration tests use (1e-3 relative).  Device memory in use (cudaMemGetInfo, which sees
+every allocation of the process, and torch's own counters) is read before and after the calls of the
+static entry point: it must not move.  Two calls matter: the built-in array is shared by all calls and keeps the
 previous call's contents, so a second call that read stale slots would show up here.  The file is named
 so that pytest collects it last.
 """
@@ -13,6 +15,7 @@ import pytest
 import torch
 
 import heatkv_workloads as W
+from oracle import heatkv_oracle as O
 
 pytestmark = pytest.mark.gpu
 
@@ -31,20 +34,47 @@ def test_static_scratch_calibration_matches_allocating_entry_point_twice():
     # all inputs exist before the calls under test: those calls must not need any allocation
     layers = [W.qkv_layer(sh, 5, l, device="cuda") for l in range(sh.L)]
     torch.cuda.synchronize()
+    # the oracle's beta of the same inputs (Eq. 2), summed over the sequences as the accumulator holds it
+    import math
+    sm = 1.0 / math.sqrt(sh.d)
+    bias_np = W.seg_bias_prior_lognormal(sh, 8)
+    ref = np.zeros((sh.L, sh.H, sh.K, sh.K))
+    for l in range(sh.L):
+        qh, kh = (O.bf16_bits_to_f64(W.bf16_bits(x)) for x in layers[l][:2])
+        for s_ in range(sh.n_seq):
+            for h in range(sh.H):
+                ref[l, h] += O.beta_sample(qh[s_, h], kh[s_, h], sh.sides, sm, bias_np[l, :, h, :].astype(np.float64))
+    # one call of each entry point first: the static one looks up its array's address on its first call, and the
+    # views / stride structs below are then the only host-side work left
+    views = []
+    for l in range(sh.L):
+        q, k, _ = layers[l]
+        for step in range(sh.K):
+            lo, hi = ses.step_slices(step)
+            qs, ks = q[:, :, lo:hi], k[:, :, :hi]
+            views.append((l, step, qs, ks, hk.Strides.of(qs, ks)))
+    warm = torch.zeros_like(want)
+    hk.heatkv_calibrate_scores_static(ses.ctx, 0, 0, sh.n_seq, views[0][2], views[0][3], views[0][4], bias[0, 0], warm)
+    torch.cuda.synchronize()
     for call in range(2):
-        for l in range(sh.L):
-            q, k, _ = layers[l]
-            for step in range(sh.K):
-                lo, hi = ses.step_slices(step)
-                qs, ks = q[:, :, lo:hi], k[:, :, :hi]
-                st = hk.Strides.of(qs, ks)
-                hk.heatkv_calibrate_scores(ses.ctx, l, step, sh.n_seq, qs, ks, None, st, bias[l, step], want, None)
-                hk.heatkv_calibrate_scores_static(ses.ctx, l, step, sh.n_seq, qs, ks, st, bias[l, step], got)
+        for (l, step, qs, ks, st) in views:
+            hk.heatkv_calibrate_scores(ses.ctx, l, step, sh.n_seq, qs, ks, None, st, bias[l, step], want, None)
         torch.cuda.synchronize()
+        free0 = torch.cuda.mem_get_info()[0]
+        torch_mem0 = (torch.cuda.memory_allocated(), torch.cuda.memory_reserved())
+        for (l, step, qs, ks, st) in views:
+            hk.heatkv_calibrate_scores_static(ses.ctx, l, step, sh.n_seq, qs, ks, st, bias[l, step], got)
+        torch.cuda.synchronize()
+        # nothing was allocated or freed on the device while the static entry point ran
+        assert torch.cuda.mem_get_info()[0] >= free0          # device-wide: an allocation of ours would lower it
+        assert (torch.cuda.memory_allocated(), torch.cuda.memory_reserved()) == torch_mem0
         a, b = want.double().cpu().numpy(), got.double().cpu().numpy()
         mask = a > 1e-5 * (call + 1)
         assert mask.sum() > 100
         assert np.all(np.abs(a - b)[mask] <= RTOL_BETA * a[mask]), (call, float(np.abs(a - b)[mask].max()))
+        r = ref * (call + 1)
+        rmask = r > 1e-5 * (call + 1)
+        assert np.all(np.abs(b - r)[rmask] <= RTOL_BETA * r[rmask]), (call, float((np.abs(b - r)[rmask] / r[rmask]).max()))
         assert np.all(np.triu(b, 1) == 0)
         # each (layer, head, step) row holds n_seq * (call + 1) probability vectors
         assert np.allclose(b.sum(axis=-1), sh.n_seq * (call + 1), atol=1e-3)
