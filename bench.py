@@ -579,6 +579,7 @@ def run_model_workload(args, which):
 
 
 def main():
+    global N_LAYERS
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
     ap.add_argument("--steps", type=int, default=50)
@@ -596,10 +597,14 @@ def main():
                          "full / larger / serving: whole-model sweeps of the other workloads; fewheads: key-range "
                          "splitting on launches with few (sequence, head) units; stability: S-CAS rank spread "
                          "over seeded calibration sets")
+    ap.add_argument("--layers", type=int, default=N_LAYERS,
+                    help="layers one step replays (default: the 2B-class model's 32; profiling runs use 1 to keep the "
+                         "device footprint small -- such a line is not the headline metric and says so in config)")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true", help="skip the host-buffer leg (profiling runs)")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
+    N_LAYERS = max(1, args.layers)
 
     rank = int(os.environ.get("RANK", "0"))
     world = int(os.environ.get("WORLD_SIZE", "1"))
