@@ -303,6 +303,12 @@ int heatkv_kernel_launches(heatkv_ctx* ctx, heatkv_kernel_stats* out);
  * of the head's rank position over the runs; 0 for the other k.  out HOST [K].  Pure host code.
  * HEATKV_ERR_NAN_SCORE if a score is not finite. */
 int heatkv_rank_dispersion(const double* scas_runs, int n_runs, int L, int H, int K, int s, double* out);
+/* Exercises the bounded wait every tensor-memory kernel uses for its hand-overs: a one-thread kernel waits,
+ * with a short limit, on a barrier that nothing will ever signal.  Synchronises `stream`.  Returns
+ * HEATKV_ERR_DEVICE_TIMEOUT when the wait gave up and set the device status word as designed (the expected
+ * outcome; the context is then in the timed-out state described above and should be destroyed), HEATKV_OK if
+ * the wait claimed success, HEATKV_ERR_CUDA on any other outcome.  Nothing faults, traps or hangs. */
+int heatkv_selftest_wait_expiry(heatkv_ctx* ctx, void* stream);
 /* Reads the device-side status word (synchronises `stream`): HEATKV_OK or
  * HEATKV_ERR_DEVICE_TIMEOUT if a bounded wait inside a kernel ran out. */
 int heatkv_device_status(heatkv_ctx* ctx, void* stream);

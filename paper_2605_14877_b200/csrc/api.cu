@@ -24,6 +24,7 @@ bool tc_supported(const TcState* st, const AttnParams& p, int d, int n_seq, bool
 cudaError_t launch_attn_tc(TcState* st, const AttnParams& p, int d, int n_seq, bool calib, cudaStream_t stream,
                            int* launches);
 int tc_split_slot_floats(int d);
+cudaError_t launch_wait_expiry(uint32_t* status, uint32_t* result, cudaStream_t stream);
 struct CalibTcState;
 uint64_t calib_tc_desc_bytes(const heatkv_config& cfg);
 int calib_tc_create(const heatkv_config& cfg, void* dev_table, cudaStream_t stream, CalibTcState** out);
@@ -1036,6 +1037,25 @@ int heatkv_rank_dispersion(const double* scas_runs, int n_runs, int L, int H, in
     return HEATKV_ERR_HOST_MEMORY;
   }
   return HEATKV_OK;
+}
+
+int heatkv_selftest_wait_expiry(heatkv_ctx* ctx, void* stream_) {
+  if (!ctx) return HEATKV_ERR_INVALID_ARG;
+  cudaStream_t stream = static_cast<cudaStream_t>(stream_);
+  // word 32 of the status region receives what the wait returned (the work counters sit in words 16 and 17)
+  uint32_t* result = ctx->status + 32;
+  if (cudaMemsetAsync(result, 0, 4, stream) != cudaSuccess) return HEATKV_ERR_CUDA;
+  if (launch_wait_expiry(ctx->status, result, stream) != cudaSuccess) return HEATKV_ERR_CUDA;
+  ctx->launches += 1;
+  ctx->kstats.other += 1;
+  uint32_t host[2] = {0, 0};
+  if (cudaMemcpyAsync(&host[0], result, 4, cudaMemcpyDeviceToHost, stream) != cudaSuccess ||
+      cudaMemcpyAsync(&host[1], ctx->status, 4, cudaMemcpyDeviceToHost, stream) != cudaSuccess ||
+      cudaStreamSynchronize(stream) != cudaSuccess)
+    return HEATKV_ERR_CUDA;
+  // the wait gave up, flagged its CTA and the context: exactly what a stuck hand-over inside a kernel does
+  if (host[0] == 2u && host[1] != 0u) return HEATKV_ERR_DEVICE_TIMEOUT;
+  return host[0] == 1u ? HEATKV_OK : HEATKV_ERR_CUDA;
 }
 
 int heatkv_device_status(heatkv_ctx* ctx, void* stream_) {

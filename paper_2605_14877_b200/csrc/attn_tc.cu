@@ -784,7 +784,26 @@ attn_tc_kernel(const __grid_constant__ AttnParams p, const __grid_constant__ Map
   }
 }
 
+// Self-test of the bounded wait: one thread waits on a barrier nobody will ever arrive at, with a short limit,
+// and reports what the wait returned.  The wait must give up, set the status word and return false.
+__global__ void wait_expiry_kernel(uint32_t* status, uint32_t* result) {
+  __shared__ __align__(8) unsigned long long barrier_word;
+  __shared__ uint32_t abort_word;
+  if (threadIdx.x == 0) {
+    abort_word = 0;
+    mbar_init(smem_u32(&barrier_word), 1);
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    const bool ok = mbar_wait(smem_u32(&barrier_word), 0, &abort_word, status, 2048u);
+    result[0] = ok ? 1u : (abort_word ? 2u : 3u);
+  }
+}
+
 }  // namespace tc
+
+cudaError_t launch_wait_expiry(uint32_t* status, uint32_t* result, cudaStream_t stream) {
+  tc::wait_expiry_kernel<<<1, 32, 0, stream>>>(status, result);
+  return cudaGetLastError();
+}
 
 // ---------------------------------------------------------------------------------- host side
 struct TcState {

@@ -24,7 +24,7 @@ __all__ = [
     "heatkv_attention_append", "heatkv_split_plan",
     "heatkv_cache_bytes", "heatkv_retained_indices", "heatkv_export_head", "heatkv_allocator_stats",
     "heatkv_launch_count", "heatkv_kernel_launches", "heatkv_rank_dispersion", "heatkv_seq_reservation", "KernelStats",
-    "heatkv_device_status", "heatkv_strerror", "heatkv_attention_split", "arena_bytes_for",
+    "heatkv_selftest_wait_expiry", "heatkv_device_status", "heatkv_strerror", "heatkv_attention_split", "arena_bytes_for",
 ]
 
 MAX_K, MAX_BATCH, PAGE_TOKENS = 16, 128, 64
@@ -102,7 +102,8 @@ def exported_symbols():
             "heatkv_scale_attention", "heatkv_attention_append", "heatkv_cache_bytes", "heatkv_seq_reservation",
             "heatkv_retained_indices", "heatkv_export_head",
             "heatkv_attention_split", "heatkv_split_plan", "heatkv_allocator_stats", "heatkv_launch_count",
-            "heatkv_kernel_launches", "heatkv_rank_dispersion", "heatkv_device_status", "heatkv_strerror"]
+            "heatkv_kernel_launches", "heatkv_rank_dispersion", "heatkv_selftest_wait_expiry", "heatkv_device_status",
+            "heatkv_strerror"]
 
 
 def _load() -> C.CDLL:
@@ -144,6 +145,7 @@ _lib.heatkv_export_head.argtypes = [_P, C.c_int, C.c_int, C.c_int, _P, _P, _P]
 _lib.heatkv_allocator_stats.argtypes = [_P, C.POINTER(AllocStats)]
 _lib.heatkv_launch_count.argtypes = [_P, C.POINTER(C.c_uint64)]
 _lib.heatkv_device_status.argtypes = [_P, _P]
+_lib.heatkv_selftest_wait_expiry.argtypes = [_P, _P]
 _lib.heatkv_kernel_launches.argtypes = [_P, C.POINTER(KernelStats)]
 _lib.heatkv_rank_dispersion.argtypes = [_P, C.c_int, C.c_int, C.c_int, C.c_int, C.c_int, _P]
 _lib.heatkv_seq_reservation.argtypes = [_P, C.c_int, C.POINTER(C.c_uint64), C.POINTER(C.c_uint64)]
@@ -367,6 +369,11 @@ def heatkv_rank_dispersion(scas_runs, s: int) -> np.ndarray:
     out = np.zeros(K, dtype=np.float64)
     _check(_lib.heatkv_rank_dispersion(_ptr(a), R, L, H, K, int(s), _ptr(out)), "heatkv_rank_dispersion")
     return out
+
+
+def heatkv_selftest_wait_expiry(ctx: int, stream=None) -> int:
+    """Status of the bounded-wait self-test: -7 (a wait ran out, as it must) is the expected answer."""
+    return _lib.heatkv_selftest_wait_expiry(ctx, _stream(stream))
 
 
 def heatkv_device_status(ctx: int, stream=None) -> int:

@@ -475,6 +475,61 @@ def test_calibration_without_output_ignores_output_strides(hk):
         assert np.allclose(outs[0], outs[1], rtol=0, atol=1e-5)
 
 
+def test_scas_stability_through_the_cuda_calibration(hk):
+    """Appendix on S-CAS stability, end to end: three seeded calibration sets through the CUDA calibration
+    (Eq. 2) -> S-CAS (Eq. 4) -> rank dispersion in the library, against the oracle's beta -> S-CAS -> dispersion
+    on the same inputs.  A head's rank must agree wherever its S-CAS is further than 2e-3 relative from both
+    neighbours in the oracle's order (closer scores may legitimately swap: the tie reading of the schedule
+    builder); when every rank agrees the dispersions are the same numbers."""
+    from paper_2605_14877_b200.sweep import Session
+    sh = W.Shape("stab", L=2, H=4, d=64, sides=W.SIDES_13[:9], n_seq=2, s=2)
+    sm = 1.0 / math.sqrt(sh.d)
+    bias = W.seg_bias_prior_lognormal(sh, 11)
+    bias_dev = torch.from_numpy(bias).cuda()
+    got_runs, ref_runs = [], []
+    for seed in (21, 22, 23):
+        with Session(sh.L, sh.H, sh.d, sh.t, sh.s, pool_rows=64, kernel=hk.KERNEL_AUTO) as ses:
+            beta_dev = torch.zeros(sh.L, sh.H, sh.K, sh.K, dtype=torch.float32, device="cuda")
+            ref = np.zeros((sh.L, sh.H, sh.K))
+            for l in range(sh.L):
+                q, k, _ = W.qkv_layer(sh, seed, l, device="cuda")
+                for step in range(sh.K):
+                    lo, hi = ses.step_slices(step)
+                    qs, ks_ = q[:, :, lo:hi], k[:, :, :hi]
+                    hk.heatkv_calibrate_scores(ses.ctx, l, step, sh.n_seq, qs, ks_, None, hk.Strides.of(qs, ks_),
+                                               bias_dev[l, step], beta_dev, None)
+                qh, kh = _f64(q), _f64(k)
+                for h in range(sh.H):
+                    b = sum(O.beta_sample(qh[s_, h], kh[s_, h], sh.sides, sm, bias[l, :, h, :].astype(np.float64))
+                            for s_ in range(sh.n_seq)) / sh.n_seq
+                    ref[l, h] = O.scas(b, sh.s)
+            _, scas, _ = hk.heatkv_finalize_scores(ses.ctx, beta_dev, sh.n_seq, sh.L, sh.H, sh.K)
+        assert np.allclose(scas, ref, rtol=RTOL_BETA, atol=1e-9)
+        got_runs.append(scas)
+        ref_runs.append(ref)
+    got_runs, ref_runs = np.stack(got_runs), np.stack(ref_runs)
+    T = sh.L * sh.H
+    all_equal = True
+    for r in range(3):
+        for kk in range(sh.s, sh.K - 1):
+            ro = O.order_from_scores(ref_runs[r].reshape(T, sh.K)[:, kk])
+            go = O.order_from_scores(got_runs[r].reshape(T, sh.K)[:, kk])
+            vals = ref_runs[r].reshape(T, sh.K)[ro, kk]
+            for pos in range(T):
+                gaps = [abs(vals[pos] - vals[j]) / max(vals[pos], 1e-30) for j in (pos - 1, pos + 1) if 0 <= j < T]
+                if min(gaps) > 2e-3:
+                    assert go[pos] == ro[pos], (r, kk, pos)
+                else:
+                    all_equal &= go[pos] == ro[pos]
+    got = hk.heatkv_rank_dispersion(got_runs, sh.s)
+    want = O.scas_rank_dispersion(ref_runs, sh.s)
+    assert np.all(got[: sh.s] == 0) and got[sh.K - 1] == 0
+    if all_equal:
+        assert np.allclose(got, want, rtol=0, atol=1e-12)
+    else:
+        assert np.allclose(got, want, rtol=0, atol=2.0 / T)
+
+
 def test_config2_all_units(hk):
     """Config 2 (2B single layer, 16 heads, d=128, 13 scales, batch 2, 20x) at full size in the
     launch configuration the bench times; the oracle checks all 32 (sequence, head) units."""
@@ -484,6 +539,21 @@ def test_config2_all_units(hk):
     bias = W.seg_bias_current_scale(sh, 0)
     _run_full_parity(hk, sh, ref, lambda ses: ses.schedule(scas=scores, b=0.05), hk.LAYOUT_PAGED, bias=bias,
                      kernel=hk.KERNEL_AUTO)                  # every one of the 32 (sequence, head) units
+
+
+def test_bounded_wait_runs_out_and_reports(hk):
+    """A hand-over that never comes: the library's self-test kernel waits (short limit) on a barrier nothing
+    signals.  The wait must end by itself, the call must answer DEVICE_TIMEOUT, the context must stay in that
+    state, and the device must go on working for other contexts."""
+    from paper_2605_14877_b200.sweep import Session
+    sh = W.Shape("expiry", L=1, H=2, d=64, sides=W.SIDES_13[:5], n_seq=1, s=1)
+    with Session(sh.L, sh.H, sh.d, sh.t, sh.s, pool_rows=256) as ses:
+        assert hk.heatkv_device_status(ses.ctx) == 0
+        assert hk.heatkv_selftest_wait_expiry(ses.ctx) == -7
+        assert hk.heatkv_device_status(ses.ctx) == -7
+    ref = O.explicit_schedule(np.ones((sh.L, sh.H)), sh.s, sh.sides)
+    _run_full_parity(hk, sh, ref, lambda ses: ses.schedule(policy=hk.POLICY_EXPLICIT, fraction=np.ones((sh.L, sh.H))),
+                     hk.LAYOUT_PAGED)
 
 
 def test_step_order_and_pool_errors(hk):

@@ -320,6 +320,19 @@ def _pieces_valid(tiles, pieces, min_piece=4):
             assert piece >= min_piece
 
 
+def test_rank_dispersion_entry_point_errors(hk):
+    runs = np.ones((2, 1, 3, 5))
+    assert np.all(hk.heatkv_rank_dispersion(runs, 1) == 0)          # equal scores: ties by head index in every run
+    bad = runs.copy()
+    bad[1, 0, 2, 2] = np.nan
+    with pytest.raises(hk.HeatKVError) as e:
+        hk.heatkv_rank_dispersion(bad, 1)
+    assert e.value.status == -6
+    with pytest.raises(hk.HeatKVError) as e:
+        hk.heatkv_rank_dispersion(runs, 5)
+    assert e.value.status == -1
+
+
 def test_split_plan_leaves_full_launches_whole():
     import paper_2605_14877_b200 as hk
     # 64 (sequence, head) units x 16 query tile pairs of equal length: 1024 items for 148 SMs, nothing to gain
