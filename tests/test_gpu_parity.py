@@ -327,7 +327,7 @@ def test_full_budget_equals_uncompressed(hk):
     _run_full_parity(hk, sh, ref, lambda ses: ses.schedule(scas=scores, b=1.0), hk.LAYOUT_PAGED)
 
 
-def _calibrate(hk, sh, seeds, bias=None, with_out=False, kernel=None):
+def _calibrate(hk, sh, seeds, bias=None, with_out=False, kernel=None, mutate=None):
     from paper_2605_14877_b200.sweep import Session
     sm = 1.0 / math.sqrt(sh.d)
     ses = Session(sh.L, sh.H, sh.d, sh.t, sh.s, pool_rows=64, kernel=hk.KERNEL_GENERIC if kernel is None else kernel)
@@ -338,6 +338,8 @@ def _calibrate(hk, sh, seeds, bias=None, with_out=False, kernel=None):
     for seed in seeds:
         for l in range(sh.L):
             q, k, v = W.qkv_layer(sh, seed, l, device="cuda")
+            if mutate is not None:
+                q, k, v = mutate(q, k, v)
             out = torch.zeros_like(q) if with_out else None
             for step in range(sh.K):
                 lo, hi = ses.step_slices(step)
@@ -407,6 +409,25 @@ def test_calibration_tensor_memory_kernel(hk, with_bias, d):
     for l in range(sh.L):
         for h in range(sh.H):
             assert np.allclose(scas[l, h], O.scas(ref[l, h], sh.s), rtol=RTOL_BETA, atol=1e-9)
+
+
+def test_calibration_tensor_memory_kernel_outlier_keys(hk):
+    """Sparse keys scaled by 16 beyond the first key tiles (logits of +-40 and more): the running reference of the
+    calibration kernel's online softmax has to move by tens of units in the middle of a row, rescaling the masses
+    parked for the finished source scales; beta must still match the oracle (Eq. 2)."""
+    sh = W.Shape("calib_outlier", L=1, H=3, d=128, sides=W.SIDES_13[:11], n_seq=2, s=3)
+
+    def mutate(q, k, v):
+        k = k.clone()
+        tok = torch.arange(k.shape[2], device=k.device)
+        pick = (tok >= 300) & (tok % 41 == 0)
+        k[:, :, pick] = k[:, :, pick] * 16
+        return q, k, v
+
+    beta, scas, cas, ref = _calibrate(hk, sh, seeds=[9], kernel=hk.KERNEL_TCGEN05, mutate=mutate)
+    mask = ref > 1e-5
+    assert np.all(np.abs(beta - ref)[mask] <= RTOL_BETA * ref[mask]), float((np.abs(beta - ref)[mask] / ref[mask]).max())
+    assert np.allclose(beta.sum(axis=-1), 1.0, atol=2e-4)
 
 
 def test_config2_calibration_full_size(hk):
