@@ -76,7 +76,7 @@ enum Bar : uint32_t {
   V_FULL = 8, V_EMPTY = 10,     // +stage
   S_FULL = 12,                  // +x  S_x of the tile is in TMEM
   P_FULL = 14,                  // +2x+h  half h (keys 64h..64h+63) of P_x of the tile is in TMEM (128 arrivals)
-  PV_DONE = 18,                 // +x  O_x includes the tile
+  PV_DONE = 18,                 // +x  O_x includes the item's last tile (one completion per item)
   ITEM_FULL = 20, ITEM_EMPTY = 22,  // +ring entry; EMPTY takes one arrival from the MMA warp and each softmax warp
   N_BARS = 24
 };
@@ -446,7 +446,7 @@ attn_tc_kernel(const __grid_constant__ AttnParams p, const __grid_constant__ Map
             tc_fence_after();
             if (leader) {
               issue_pv(x, st, 1, false);
-              tc_commit(bar(PV_DONE + x));
+              if (!more) tc_commit(bar(PV_DONE + x));                   // only the epilogue waits for it
             }
             __syncwarp();
             if (more) {
@@ -508,6 +508,7 @@ attn_tc_kernel(const __grid_constant__ AttnParams p, const __grid_constant__ Map
     unsigned char* stage = sgen + SM_OUT + (warp - 4) * STAGE_BYTES;
     const float LOG2E = 1.4426950408889634f;
     uint32_t cx = 0;                                    // key tiles of this query tile so far (all items)
+    uint32_t items_x = 0;                               // items in which this query tile held rows so far
     bool ok = true;
     for (uint32_t it = 0; ok; ++it) {
       const uint32_t slot = it & 1;
@@ -582,10 +583,9 @@ attn_tc_kernel(const __grid_constant__ AttnParams p, const __grid_constant__ Map
             const float m_new = fmaxf(m_ref, mx);
             const bool grow = m_new > m_ref + RESCALE_THRESHOLD;   // also true on the first tile (m_ref = -inf)
             if (j > 0 && __any_sync(0xffffffffu, grow)) {
-              // O_x holds tiles < j relative to m_ref: rescale the rows whose reference moves
-              ok = __all_sync(0xffffffffu, mbar_wait(bar(PV_DONE + x), ph ^ 1, abort_flag, p.status));
-              if (!ok) break;
-              tc_fence_after();
+              // O_x holds tiles < j relative to m_ref: rescale the rows whose reference moves.  O_x is complete:
+              // S_x of this tile was issued after the PV products of tile j - 1 by the same thread, and the
+              // commit behind S_FULL covers every product issued before it.
               const float f = grow ? exp2f(m_ref - m_new) : 1.f;
 #pragma unroll
               for (int c = 0; c < D / 32; ++c) {
@@ -641,7 +641,8 @@ attn_tc_kernel(const __grid_constant__ AttnParams p, const __grid_constant__ Map
             tc_fence_before();
             mbar_arrive(bar(P_FULL + 2 * x + 1));
           }
-          if (ok) ok = __all_sync(0xffffffffu, mbar_wait(bar(PV_DONE + x), (cx + n_tiles - 1) & 1, abort_flag, p.status));
+          if (ok) ok = __all_sync(0xffffffffu, mbar_wait(bar(PV_DONE + x), items_x & 1, abort_flag, p.status));
+          ++items_x;
           cx += n_tiles;
           const Item im = read_item(ring, p, n_qp);
           const int seq = im.seq;
