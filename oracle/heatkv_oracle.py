@@ -17,7 +17,10 @@ Readings taken where the paper is silent or ambiguous (each is also listed in th
 design notes): see `cache_size_after_layer` (physical vs. literal future-layer
 accounting), `budget_tokens` (integer budget), `order_from_scores` (tie order),
 `heatkv_schedule` (last step), `explicit_schedule` (per-head fraction policy, which
-has no counterpart in the paper: parity unpinned).
+has no counterpart in the paper: parity unpinned), and the fp8 cache format at the end of
+the file (`quantize_rows_e4m3` / `dequantize_rows_e4m3`: the paper only points at
+quantisation, so the format is this library's own: parity unpinned by the paper; the
+rounding itself is pinned to the published E4M3 encoding and to a library conversion).
 """
 from __future__ import annotations
 
@@ -417,3 +420,76 @@ def scas_rank_dispersion(scas_runs: np.ndarray, s: int) -> np.ndarray:
             acc += var ** 0.5
         out[k - 1] = acc / T
     return out
+
+
+# ----------------------------------------------------------------------------- fp8 K/V cache (build-defined)
+# The paper names cache quantisation only as an orthogonal direction (Sec. 5 and the conclusion) and defines
+# no format, so everything below is this library's own definition: PARITY UNPINNED BY THE PAPER.  What the
+# format borrows is public: the 8-bit E4M3 encoding of the OCP "8-bit floating point" specification
+# (1 sign, 4 exponent bits with bias 7, 3 mantissa bits; subnormals; no infinities; S.1111.111 is NaN;
+# largest finite value 448), and power-of-two block scales as in microscaling formats.
+#
+# A cached row (the d values of one token of one head, K or V) is stored as d E4M3 codes plus one signed
+# byte e: code_j = RN_even_E4M3(x_j * 2^-e), where e is the smallest integer >= FP8_EXP_MIN with
+# max_j |x_j| * 2^-e <= 448.  Reading the cache gives x^_j = value(code_j) * 2^e, which a bf16 holds exactly;
+# attention then runs on x^ exactly as it does on an unquantised cache.
+FP8_EXP_MIN = -120
+FP8_MAX = 448.0
+
+
+def e4m3_values() -> np.ndarray:
+    """value[code] for the 256 E4M3 codes, from the format's definition (NaN for 0x7f and 0xff)."""
+    out = np.zeros(256, dtype=np.float64)
+    for code in range(256):
+        sign = -1.0 if code & 0x80 else 1.0
+        ex, man = (code >> 3) & 0xF, code & 0x7
+        if ex == 0xF and man == 0x7:
+            out[code] = np.nan
+        elif ex == 0:
+            out[code] = sign * (man / 8.0) * 2.0 ** (-6)
+        else:
+            out[code] = sign * (1.0 + man / 8.0) * 2.0 ** (ex - 7)
+    return out
+
+
+def fp8_row_exponents(x: np.ndarray) -> np.ndarray:
+    """[n] the exponent byte of every row of x [n, d] (finite values)."""
+    amax = np.abs(x).max(axis=1)
+    e = np.full(x.shape[0], FP8_EXP_MIN, dtype=np.int64)
+    for r in range(x.shape[0]):
+        a = float(amax[r])
+        if a == 0.0:
+            continue
+        k = int(np.ceil(np.log2(a / FP8_MAX))) - 2      # start below the answer, then walk up exactly
+        while a * 2.0 ** (-k) > FP8_MAX:
+            k += 1
+        e[r] = max(k, FP8_EXP_MIN)
+    return e
+
+
+def quantize_rows_e4m3(x: np.ndarray):
+    """x [n, d] float64 (bf16 values widened exactly) -> (codes uint8 [n, d], exps int8 [n]).
+    Round to nearest on the E4M3 grid, ties to the code with an even mantissa; zero keeps its sign."""
+    vals = e4m3_values()
+    pos = vals[:0x7F]                                     # codes 0 .. 0x7e ascend from 0 to 448
+    e = fp8_row_exponents(x)
+    y = x * np.exp2(-e.astype(np.float64))[:, None]       # exact: a power-of-two scaling
+    a = np.abs(y)
+    hi = np.searchsorted(pos, a, side="left")             # first code with value >= a
+    hi = np.minimum(hi, 0x7E)
+    lo = np.maximum(hi - 1, 0)
+    d_hi, d_lo = pos[hi] - a, a - pos[lo]
+    take_lo = (d_lo < d_hi) | ((d_lo == d_hi) & (lo % 2 == 0))
+    code = np.where(take_lo, lo, hi).astype(np.uint8)
+    code = np.where(np.signbit(y), code | 0x80, code).astype(np.uint8)
+    return code, e.astype(np.int8)
+
+
+def dequantize_rows_e4m3(codes: np.ndarray, exps: np.ndarray) -> np.ndarray:
+    """[n, d] float64: value(code) * 2^e, exactly."""
+    return e4m3_values()[codes] * np.exp2(exps.astype(np.float64))[:, None]
+
+
+def cache_bytes_fp8(kept: np.ndarray, d: int) -> int:
+    """sum over (layer, head) of kept_tokens * (head_dim codes + 1 exponent byte) * 2 (K and V)."""
+    return int(kept.sum()) * (d + 1) * 2

@@ -474,3 +474,71 @@ def test_scas_rank_dispersion_pins():
     assert np.isclose(d[k], 2 * 0.5 / (L * H))
     assert np.all(d[:s] == 0) and d[K - 1] == 0
     assert np.all(np.delete(d, k) == 0)
+
+
+# ----------------------------------------------------------------------------- fp8 cache format (build-defined)
+def _fp8_golden_rows():
+    rows = []
+    for raw in open(os.path.join(GOLDEN, "fp8_rows.txt")):
+        line = raw.split("#")[0].strip()
+        if not line:
+            continue
+        a, b, c = line.split(":")
+        rows.append((int(a.split()[1]), [float(v) for v in b.split()], [int(v, 16) for v in c.split()]))
+    return rows
+
+
+def test_fp8_rows_hand_worked():
+    """Exponent byte and E4M3 codes of the rows derived by hand in tests/golden/fp8_rows.txt (ties to even,
+    subnormals, signed zero, the exact-fit exponent)."""
+    for e, x, codes in _fp8_golden_rows():
+        got_c, got_e = O.quantize_rows_e4m3(np.array([x], dtype=np.float64))
+        assert int(got_e[0]) == e
+        assert [int(v) for v in got_c[0]] == codes
+
+
+def test_e4m3_table_closed_forms():
+    """The code table against the format's closed forms: 0x38 = 1, 0x7e = 448 (largest finite), 0x08 = 2^-6
+    (smallest normal), 0x01 = 2^-9 (smallest subnormal), NaN only at S.1111.111, odd symmetry, strictly
+    ascending positive half."""
+    v = O.e4m3_values()
+    assert v[0x38] == 1.0 and v[0x7E] == 448.0 and v[0x08] == 2.0 ** -6 and v[0x01] == 2.0 ** -9 and v[0] == 0.0
+    assert np.isnan(v[0x7F]) and np.isnan(v[0xFF]) and np.isnan(v).sum() == 2
+    assert (np.diff(v[:0x7F]) > 0).all()
+    assert (v[0x80:0xFF] == -v[0x00:0x7F]).all()
+
+
+def test_fp8_quantiser_matches_a_library_conversion():
+    """Inside the finite range the rounding is the one of a library float32 -> float8_e4m3fn conversion
+    (round to nearest even); the row exponent is minimal; the read-back value is exactly a bf16; reading and
+    quantising again changes no value; the error stays below half a grid step."""
+    import torch
+    rng = np.random.default_rng(7)
+    x = rng.standard_normal((96, 128)) * np.exp2(rng.integers(-30, 30, (96, 1)).astype(np.float64))
+    x[5] = 0.0
+    x[6, :] = 448.0 * 2.0 ** 3
+    x[7, 3] = -x[7].max() * 4
+    x = torch.from_numpy(x).to(torch.bfloat16).to(torch.float64).numpy()          # exactly bf16 values
+    codes, e = O.quantize_rows_e4m3(x)
+    y = x * np.exp2(-e.astype(np.float64))[:, None]
+    amax = np.abs(y).max(axis=1)
+    assert (amax <= 448.0).all()
+    nz = np.abs(x).max(axis=1) > 0
+    assert ((amax[nz] * 2 > 448.0) | (e[nz] == O.FP8_EXP_MIN)).all()              # e - 1 would not fit
+    lib = torch.from_numpy(y).to(torch.float32).to(torch.float8_e4m3fn).view(torch.uint8).numpy()
+    assert (lib == codes).all()
+    xh = O.dequantize_rows_e4m3(codes, e)
+    assert (torch.from_numpy(xh).to(torch.bfloat16).to(torch.float64).numpy() == xh).all()
+    c2, e2 = O.quantize_rows_e4m3(xh)
+    assert (O.dequantize_rows_e4m3(c2, e2) == xh).all()
+    # half a step of the grid at the row's largest value: 2^(e + 8 - 3) / 2
+    assert (np.abs(xh - x) <= np.exp2(e.astype(np.float64) + 4)[:, None]).all()
+    # elementwise: relative error at most 2^-4 for values in the normal range of the scaled grid
+    normal = np.abs(y) >= 2.0 ** -6
+    assert (np.abs(xh - x)[normal] <= np.abs(x)[normal] * 2.0 ** -4).all()
+
+
+def test_fp8_cache_bytes_closed_form():
+    kept = np.array([[10, 0], [7, 3]])
+    assert O.cache_bytes_fp8(kept, 128) == 20 * 129 * 2
+    assert O.cache_bytes_fp8(kept, 128) * 2 < O.cache_bytes(kept, 128) * 1.01 + 1
