@@ -75,6 +75,11 @@ typedef enum {
   HEATKV_KERNEL_TCGEN05 = 2    /* tcgen05 / TMEM / TMA kernel wherever its shape rules allow */
 } heatkv_kernel_choice;
 
+typedef enum {
+  HEATKV_CACHE_BF16 = 0,       /* rows stored verbatim                                            */
+  HEATKV_CACHE_FP8_E4M3 = 1    /* rows stored as 8-bit codes plus one exponent byte (see below)    */
+} heatkv_cache_dtype;
+
 typedef struct heatkv_ctx heatkv_ctx;
 typedef struct heatkv_schedule heatkv_schedule;
 
@@ -91,6 +96,10 @@ typedef struct {
   uint64_t scratch_bytes;        /* bytes of the arena for partial results of heads whose key range is
                                     split over several CTAs; 0 = default (1/8 of the arena, at most
                                     128 MiB); too little only disables splitting                    */
+  int32_t cache_dtype;           /* heatkv_cache_dtype; FP8_E4M3 needs the paged layout                    */
+  int32_t reserved0;
+  uint64_t stage_bytes;          /* FP8_E4M3 only: bytes of the arena for the bf16 staging rows one attention
+                                    call expands its visible keys into; 0 = default (1/8 of the arena)     */
 } heatkv_config;
 
 typedef struct {                 /* element strides of the [n_seq, H, t, d] activations    */
@@ -120,7 +129,24 @@ typedef struct {
   uint32_t plans;                /* schedules whose plan is resident                        */
 } heatkv_alloc_stats;
 
-/* Context: validates the shape, splits the arena into a metadata region and the K / V
+/* fp8 cache (cache_dtype = HEATKV_CACHE_FP8_E4M3).  The paper names quantisation of the cache only as an
+ * orthogonal direction (Sec. 5 and the conclusion) and defines no format; this one is the library's own.
+ * A cached row (the d values of one token of one head, K or V) is stored as d codes of the OCP 8-bit
+ * floating-point format E4M3 (1 sign, 4 exponent bits with bias 7, 3 mantissa bits, subnormals, no
+ * infinities, largest finite value 448) plus one signed exponent byte e:
+ *     code_j = round-to-nearest-even on the E4M3 grid of x_j * 2^-e,
+ *     e = the smallest integer >= -120 with max_j |x_j| * 2^-e <= 448   (all-zero row: e = -120),
+ * so a row costs d + 1 bytes instead of 2 d.  Reading gives x^_j = value(code_j) * 2^e, which a bf16 holds
+ * exactly.  Attention in such a context is attention over x^ for the cached scales (the step's own K/V come
+ * from k_new / v_new unquantised, as always): before the attention kernel runs, the call expands the visible
+ * head-scales of its (layer, step) into bf16 staging rows inside the arena (stage_bytes), and the attention
+ * kernels read those; the update after the layer quantises the new rows on their way into the pool.  Inputs
+ * must be finite.  Only the paged layout is supported; heatkv_attention_append issues its parts as separate
+ * kernels in such a context.  A call whose sequences need more staging rows than stage_bytes holds returns
+ * HEATKV_ERR_OUT_OF_PAGES (rows needed per sequence: the largest number of visible 64-row half-tiles of any
+ * (layer, step) of its schedule, times 64).
+ *
+ * Context: validates the shape, splits the arena into a metadata region and the K / V
  * pools, zero-fills the pools (enqueued on `stream`).  The arena must outlive the context.
  * With kernel = HEATKV_KERNEL_AUTO or HEATKV_KERNEL_TCGEN05 the tensor-memory kernels are set up here; if that
  * fails on a device of compute capability 10.x (or on any device under HEATKV_KERNEL_TCGEN05) the call returns
@@ -277,7 +303,8 @@ int heatkv_split_plan(const int32_t* tiles /*HOST*/, int n_heads, int n_qp, int 
                       double* makespan_cut);
 
 /* Introspection (host state only unless noted). */
-/* Bytes of K and V the sequence holds right now, two ways: *actual = the pool rows its plan has placed for the
+/* (With the fp8 cache a row counts d + 1 bytes instead of 2 d in both figures.)
+ * Bytes of K and V the sequence holds right now, two ways: *actual = the pool rows its plan has placed for the
  * head-scales it stores (valid rows of their destination half-tiles) x d x 2 (K and V) x 2 bytes; *closed_form =
  * sum over (layer, head) of kept_tokens x d x 2 x 2 from the schedule's masks (Sec. 3.2: the cache size in
  * tokens).  The two agree unless the plan and the schedule have come apart.  Either may be NULL. */
@@ -291,6 +318,11 @@ int heatkv_retained_indices(heatkv_ctx* ctx, int seq_id, int layer, int head, in
  * n*d bf16 each (enqueued on `stream`). */
 int heatkv_export_head(heatkv_ctx* ctx, int seq_id, int layer, int head, void* k_out, void* v_out,
                        void* stream);
+/* The same for a context with the fp8 cache (heatkv_export_head answers HEATKV_ERR_INVALID_ARG there, and this
+ * call in a bf16 context): the head's n cached rows in logical order as stored, k_codes / v_codes DEVICE
+ * uint8 [n][d] (E4M3 codes) and k_exps / v_exps DEVICE int8 [n] (the rows' exponent bytes). */
+int heatkv_export_head_fp8(heatkv_ctx* ctx, int seq_id, int layer, int head, void* k_codes, void* v_codes,
+                           void* k_exps, void* v_exps, void* stream);
 int heatkv_allocator_stats(heatkv_ctx* ctx, heatkv_alloc_stats* out);
 /* Kernels launched by this context so far. */
 int heatkv_launch_count(heatkv_ctx* ctx, uint64_t* n);

@@ -16,6 +16,8 @@ cudaError_t launch_attn_generic(const AttnParams& p, int d, int n_seq, bool cali
 cudaError_t launch_calibrate_static(const AttnParams& p, int d, int n_seq, cudaStream_t stream, bool* too_large);
 cudaError_t launch_append(const CopyParams& p, int n_seq, cudaStream_t stream);
 cudaError_t launch_compact(const CopyParams& p, int n_seq, cudaStream_t stream);
+cudaError_t launch_append_fp8(const CopyParams& p, int n_seq, cudaStream_t stream);
+cudaError_t launch_dequant_fp8(const CopyParams& p, int n_seq, int slots, cudaStream_t stream);
 struct TcState;
 int tc_create(const heatkv_config& cfg, void* k_pool, void* v_pool, uint64_t pool_rows, TcState** out);
 void tc_destroy(TcState* st);
@@ -111,6 +113,14 @@ struct heatkv_ctx {
   __nv_bfloat16* k_pool = nullptr;
   __nv_bfloat16* v_pool = nullptr;
   uint64_t pool_rows = 0, meta_bytes = 0;
+  // fp8 cache: k_pool / v_pool above are then the bf16 staging rows the attention kernels read (stage_rows of
+  // them), and the cache proper is these code pools [pool_rows][d] with one exponent byte per row
+  bool fp8 = false;
+  uint8_t* k8_pool = nullptr;
+  uint8_t* v8_pool = nullptr;
+  int8_t* k_exp = nullptr;
+  int8_t* v_exp = nullptr;
+  uint64_t stage_rows = 0;
   uint32_t* status = nullptr;
   RangeAlloc rows, metas;
   std::vector<std::unique_ptr<PlanEntry>> plans;
@@ -141,7 +151,7 @@ int find_or_load_plan(heatkv_ctx* ctx, const Schedule& s, cudaStream_t stream, i
   if (!e) return HEATKV_ERR_HOST_MEMORY;
   e->uid = s.uid;
   e->sched = s;
-  int rc = build_plan(s, ctx->cfg.layout, &e->plan);
+  int rc = build_plan(s, ctx->cfg.layout, &e->plan, ctx->fp8);
   if (rc != HEATKV_OK) return rc;
   uint64_t bytes = ((uint64_t)e->plan.blob.size() * 4 + META_ALIGN - 1) / META_ALIGN * META_ALIGN;
   uint64_t off = 0;
@@ -380,6 +390,9 @@ int heatkv_create(const heatkv_config* cfg, void* stream_, heatkv_ctx** out) {
   if (cfg->s < 0 || cfg->s > (cfg->K > 1 ? cfg->K - 1 : 0)) return HEATKV_ERR_INVALID_ARG;
   if (cfg->layout != HEATKV_LAYOUT_RAGGED && cfg->layout != HEATKV_LAYOUT_PAGED) return HEATKV_ERR_INVALID_ARG;
   if (cfg->kernel < HEATKV_KERNEL_AUTO || cfg->kernel > HEATKV_KERNEL_TCGEN05) return HEATKV_ERR_INVALID_ARG;
+  if (cfg->cache_dtype != HEATKV_CACHE_BF16 && cfg->cache_dtype != HEATKV_CACHE_FP8_E4M3) return HEATKV_ERR_INVALID_ARG;
+  const bool fp8 = cfg->cache_dtype == HEATKV_CACHE_FP8_E4M3;
+  if (fp8 && cfg->layout != HEATKV_LAYOUT_PAGED) return HEATKV_ERR_INVALID_ARG;
   if (!cfg->arena || (reinterpret_cast<uintptr_t>(cfg->arena) & 1023)) return HEATKV_ERR_INVALID_ARG;
   for (int i = 0; i < cfg->K; ++i)
     if (cfg->t[i] < 1 || cfg->t[i] > (1 << 20)) return HEATKV_ERR_INVALID_ARG;
@@ -398,11 +411,25 @@ int heatkv_create(const heatkv_config* cfg, void* stream_, heatkv_ctx** out) {
   scratch = (scratch + 1023) / 1024 * 1024;
   if (cfg->arena_bytes < meta + scratch + 2ull * HEATKV_PAGE_TOKENS * cfg->d * 2) return HEATKV_ERR_INVALID_ARG;
   const uint64_t row_bytes = (uint64_t)cfg->d * 2;
-  uint64_t rows = (cfg->arena_bytes - meta - scratch) / (2 * row_bytes);
+  // bf16 cache: the rest of the arena is the K pool and the V pool.  fp8 cache: first the bf16 staging rows
+  // (K and V), then the two code pools and the two exponent arrays.
+  uint64_t stage_rows = 0, rows = 0;
+  if (fp8) {
+    uint64_t stage = cfg->stage_bytes ? cfg->stage_bytes : cfg->arena_bytes / 8;
+    stage_rows = stage / (2 * row_bytes) / HEATKV_PAGE_TOKENS * HEATKV_PAGE_TOKENS;
+    if (stage_rows > 0x7fffffc0ull) stage_rows = 0x7fffffc0ull;
+    const uint64_t used = meta + scratch + 2 * stage_rows * row_bytes;
+    if (stage_rows == 0 || cfg->arena_bytes < used + 2ull * HEATKV_PAGE_TOKENS * (cfg->d + 1)) return HEATKV_ERR_INVALID_ARG;
+    rows = (cfg->arena_bytes - used) / (2ull * (cfg->d + 1));
+  } else {
+    rows = (cfg->arena_bytes - meta - scratch) / (2 * row_bytes);
+  }
   rows = rows / HEATKV_PAGE_TOKENS * HEATKV_PAGE_TOKENS;
   if (rows > 0x7fffffffull) rows = 0x7fffffc0ull;
   ctx->meta = static_cast<unsigned char*>(cfg->arena);
   ctx->meta_bytes = meta;
+  ctx->fp8 = fp8;
+  ctx->stage_rows = stage_rows;
   ctx->k_pool = reinterpret_cast<__nv_bfloat16*>(ctx->meta + meta + scratch);
   {   // scratch region: arrival counters first (kept zero between launches), then the partial-result slots
     const uint64_t ctr_bytes = std::min<uint64_t>(scratch / 4, 256u << 10) / 1024 * 1024;
@@ -417,16 +444,24 @@ int heatkv_create(const heatkv_config* cfg, void* stream_, heatkv_ctx** out) {
         cudaDeviceGetAttribute(&n_sm, cudaDevAttrMultiProcessorCount, dev) == cudaSuccess && n_sm > 0)
       ctx->n_sm = n_sm;
   }
-  ctx->v_pool = ctx->k_pool + rows * cfg->d;
+  const uint64_t bf16_rows = fp8 ? stage_rows : rows;           // rows of the two bf16 arrays the attention kernels read
+  ctx->v_pool = ctx->k_pool + bf16_rows * cfg->d;
   ctx->pool_rows = rows;
+  if (fp8) {
+    ctx->k8_pool = reinterpret_cast<uint8_t*>(ctx->v_pool + bf16_rows * cfg->d);
+    ctx->v8_pool = ctx->k8_pool + rows * cfg->d;
+    ctx->k_exp = reinterpret_cast<int8_t*>(ctx->v8_pool + rows * cfg->d);
+    ctx->v_exp = ctx->k_exp + rows;
+  }
   ctx->status = reinterpret_cast<uint32_t*>(ctx->meta);
   ctx->rows.reset(0, rows);
   ctx->metas.reset(STATUS_BYTES, meta - STATUS_BYTES);
   // zero the status word and both pools: half-tiles are read whole, rows past a tile's valid
   // count must hold finite values
   if (cudaMemsetAsync(ctx->meta, 0, STATUS_BYTES, stream) != cudaSuccess) return HEATKV_ERR_CUDA;
-  if (cudaMemsetAsync(ctx->k_pool, 0, 2 * rows * row_bytes, stream) != cudaSuccess) return HEATKV_ERR_CUDA;
-  int rc = tc_create(ctx->cfg, ctx->k_pool, ctx->v_pool, rows, &ctx->tc);
+  if (cudaMemsetAsync(ctx->k_pool, 0, 2 * bf16_rows * row_bytes, stream) != cudaSuccess) return HEATKV_ERR_CUDA;
+  if (fp8 && cudaMemsetAsync(ctx->k8_pool, 0, 2 * rows * ((uint64_t)cfg->d + 1), stream) != cudaSuccess) return HEATKV_ERR_CUDA;
+  int rc = tc_create(ctx->cfg, ctx->k_pool, ctx->v_pool, bf16_rows, &ctx->tc);
   if (rc != HEATKV_OK) {
     tc_destroy(ctx->tc);
     return rc;
@@ -605,7 +640,37 @@ static int attention_impl(heatkv_ctx* ctx, const int* seq_ids, int n_seq, int la
   bool use_tc = choice != HEATKV_KERNEL_GENERIC && tc_supported(ctx->tc, p, ctx->cfg.d, n_seq, false);
   if (choice == HEATKV_KERNEL_AUTO && p.t_q < 256) use_tc = false;
   if (choice == HEATKV_KERNEL_TCGEN05 && !use_tc) return HEATKV_ERR_INVALID_ARG;   // never a silent substitute
-  bool fuse = with_update && stores && ctx->cfg.layout == HEATKV_LAYOUT_PAGED;
+  if (ctx->fp8) {
+    // The attention kernels read bf16 rows: expand the visible head-scales of this (layer, step) from the code
+    // pools into the staging rows first (every sequence gets the rows its plan needs, one after the other),
+    // then point the kernels' row numbering at them.
+    CopyParams cp;
+    std::memset(&cp, 0, sizeof(cp));
+    cp.k_pool = ctx->k_pool; cp.v_pool = ctx->v_pool;
+    cp.k8_pool = ctx->k8_pool; cp.v8_pool = ctx->v8_pool; cp.k_exp = ctx->k_exp; cp.v_exp = ctx->v_exp;
+    cp.step = step; cp.layer = layer; cp.H = ctx->cfg.H; cp.K = ctx->cfg.K; cp.L = ctx->cfg.L; cp.d = ctx->cfg.d;
+    uint64_t next = 0;
+    int slots = 0;
+    for (int i = 0; i < n_seq; ++i) {
+      const PlanEntry& pe = *ctx->plans[ctx->seqs[seq_ids[i]].plan];
+      const PlanHeader& hd = pe.plan.header();
+      const int32_t* blob = pe.plan.blob.data();
+      const size_t u0 = pe.sched.at(step, layer, 0), u1 = pe.sched.at(step, layer, pe.sched.H - 1);
+      const int count = blob[hd.off_attn_begin + u1] + blob[hd.off_attn_cnt + u1] - blob[hd.off_attn_begin + u0];
+      slots = std::max(slots, count);
+      cp.seqs[i] = p.seqs[i];
+      cp.stage_base[i] = (int32_t)next;
+      next += (uint64_t)count * HEATKV_PAGE_TOKENS;
+    }
+    if (next > ctx->stage_rows) return HEATKV_ERR_OUT_OF_PAGES;
+    if (launch_dequant_fp8(cp, n_seq, slots, stream) != cudaSuccess) return HEATKV_ERR_CUDA;
+    if (slots > 0) {
+      ctx->launches += 1;
+      ctx->kstats.other += 1;
+    }
+    for (int i = 0; i < n_seq; ++i) p.seqs[i].base_row = cp.stage_base[i];
+  }
+  bool fuse = with_update && stores && ctx->cfg.layout == HEATKV_LAYOUT_PAGED && !ctx->fp8;
   if (fuse) {
     // The tensor-memory kernel copies the new rows with two spare warps per SM beside the attention work, so
     // the update rides along whatever its size.  The generic kernel carries it as extra CTAs of its own
@@ -860,7 +925,8 @@ int heatkv_append_compact(heatkv_ctx* ctx, const int* seq_ids, int n_seq, int la
         ctx->kstats.compact += 1;
       }
     }
-    if (launch_append(p, n_seq, stream) != cudaSuccess) return HEATKV_ERR_CUDA;
+    p.k8_pool = ctx->k8_pool; p.v8_pool = ctx->v8_pool; p.k_exp = ctx->k_exp; p.v_exp = ctx->v_exp;
+    if ((ctx->fp8 ? launch_append_fp8(p, n_seq, stream) : launch_append(p, n_seq, stream)) != cudaSuccess) return HEATKV_ERR_CUDA;
     ctx->launches += 1;
     ctx->kstats.append += 1;
   }
@@ -890,8 +956,9 @@ int heatkv_cache_bytes(heatkv_ctx* ctx, int seq_id, uint64_t* actual, uint64_t* 
         for (int j = 0; j < cnt; ++j) placed += descs[b0 + j].meta & 0xff;
       }
     }
-  if (actual) *actual = placed * ctx->cfg.d * 2 * 2;
-  if (closed_form) *closed_form = tokens * ctx->cfg.d * 2 * 2;
+  const uint64_t row_bytes = ctx->fp8 ? (uint64_t)ctx->cfg.d + 1 : (uint64_t)ctx->cfg.d * 2;   // per row of K or of V
+  if (actual) *actual = placed * row_bytes * 2;
+  if (closed_form) *closed_form = tokens * row_bytes * 2;
   return HEATKV_OK;
 }
 
@@ -922,7 +989,7 @@ int heatkv_retained_indices(heatkv_ctx* ctx, int seq_id, int layer, int head, in
 }
 
 int heatkv_export_head(heatkv_ctx* ctx, int seq_id, int layer, int head, void* k_out, void* v_out, void* stream_) {
-  if (!ctx || !k_out || !v_out) return HEATKV_ERR_INVALID_ARG;
+  if (!ctx || !k_out || !v_out || ctx->fp8) return HEATKV_ERR_INVALID_ARG;
   Seq* q = get_seq(ctx, seq_id);
   if (!q || layer < 0 || layer >= ctx->cfg.L || head < 0 || head >= ctx->cfg.H) return HEATKV_ERR_INVALID_ARG;
   cudaStream_t stream = static_cast<cudaStream_t>(stream_);
@@ -966,6 +1033,44 @@ int heatkv_export_head(heatkv_ctx* ctx, int seq_id, int layer, int head, void* k
   return HEATKV_OK;
 }
 
+int heatkv_export_head_fp8(heatkv_ctx* ctx, int seq_id, int layer, int head, void* k_codes, void* v_codes, void* k_exps,
+                           void* v_exps, void* stream_) {
+  if (!ctx || !k_codes || !v_codes || !k_exps || !v_exps || !ctx->fp8) return HEATKV_ERR_INVALID_ARG;
+  Seq* q = get_seq(ctx, seq_id);
+  if (!q || layer < 0 || layer >= ctx->cfg.L || head < 0 || head >= ctx->cfg.H) return HEATKV_ERR_INVALID_ARG;
+  cudaStream_t stream = static_cast<cudaStream_t>(stream_);
+  const PlanEntry& pe = *ctx->plans[q->plan];
+  const Schedule& s = pe.sched;
+  const PlanHeader& h = pe.plan.header();
+  const int32_t* blob = pe.plan.blob.data();
+  const Desc* descs = reinterpret_cast<const Desc*>(blob + h.off_desc);
+  const uint16_t m = stored_mask(ctx, *q, layer, head);
+  const size_t d = (size_t)ctx->cfg.d;
+  size_t out_row = 0;
+  for (int i = 0; i < s.K; ++i) {
+    if (!((m >> i) & 1)) continue;
+    // a head-scale keeps the rows it was appended to for its whole life (append descriptors carry pool rows)
+    const size_t u = s.at(i, layer, head);
+    const int32_t b0 = blob[h.off_app_begin + u], cnt = blob[h.off_app_cnt + u];
+    for (int j = 0; j < cnt; ++j) {
+      const Desc& dsc = descs[b0 + j];
+      const size_t nrow = (size_t)(dsc.meta & 0xff);
+      const int64_t row = (int64_t)q->base_row + dsc.row;
+      if (cudaMemcpyAsync(static_cast<char*>(k_codes) + out_row * d, ctx->k8_pool + row * d, nrow * d,
+                          cudaMemcpyDeviceToDevice, stream) != cudaSuccess ||
+          cudaMemcpyAsync(static_cast<char*>(v_codes) + out_row * d, ctx->v8_pool + row * d, nrow * d,
+                          cudaMemcpyDeviceToDevice, stream) != cudaSuccess ||
+          cudaMemcpyAsync(static_cast<char*>(k_exps) + out_row, ctx->k_exp + row, nrow, cudaMemcpyDeviceToDevice,
+                          stream) != cudaSuccess ||
+          cudaMemcpyAsync(static_cast<char*>(v_exps) + out_row, ctx->v_exp + row, nrow, cudaMemcpyDeviceToDevice,
+                          stream) != cudaSuccess)
+        return HEATKV_ERR_CUDA;
+      out_row += nrow;
+    }
+  }
+  return HEATKV_OK;
+}
+
 int heatkv_allocator_stats(heatkv_ctx* ctx, heatkv_alloc_stats* out) {
   if (!ctx || !out) return HEATKV_ERR_INVALID_ARG;
   std::memset(out, 0, sizeof(*out));
@@ -978,7 +1083,7 @@ int heatkv_allocator_stats(heatkv_ctx* ctx, heatkv_alloc_stats* out) {
       out->open_seqs++;
       uint64_t bytes = 0;
       heatkv_cache_bytes(ctx, (int)i, nullptr, &bytes);
-      out->used_tokens += bytes / ((uint64_t)ctx->cfg.d * 4);
+      out->used_tokens += bytes / (ctx->fp8 ? ((uint64_t)ctx->cfg.d + 1) * 2 : (uint64_t)ctx->cfg.d * 4);
     }
   for (auto& pe : ctx->plans)
     if (pe) out->plans++;

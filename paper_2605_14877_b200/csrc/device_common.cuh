@@ -68,6 +68,13 @@ struct CopyParams {
   int32_t phase;                  // compaction: 0 = before the step, 1 = after the layer
   int32_t layer_begin, n_layers;  // compaction before a step may cover all layers
   SeqRef seqs[HEATKV_MAX_BATCH];
+  // ---- fp8 cache: code pools [rows][d], one exponent byte per row, and the first staging row of every
+  // sequence of the call (the bf16 staging rows are k_pool / v_pool)
+  uint8_t* k8_pool;
+  uint8_t* v8_pool;
+  int8_t* k_exp;
+  int8_t* v_exp;
+  int32_t stage_base[HEATKV_MAX_BATCH];
 };
 
 // ---- plan blob accessors (see PlanHeader in internal.h: word offsets from the blob start)
@@ -88,6 +95,7 @@ struct PlanView {
   __device__ __forceinline__ const int32_t* pre_cnt() const { return w + w[12]; }
   __device__ __forceinline__ const int32_t* post_begin() const { return w + w[13]; }
   __device__ __forceinline__ const int32_t* post_cnt() const { return w + w[14]; }
+  __device__ __forceinline__ const int32_t* src_rows() const { return w + w[17]; }   // fp8 cache only
 };
 
 __device__ __forceinline__ uint32_t smem_u32(const void* p) {

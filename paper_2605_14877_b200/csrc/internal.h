@@ -49,7 +49,9 @@ struct PlanHeader {
   int32_t off_post_cnt;
   int32_t n_move;
   int32_t total_words;
-  int32_t pad[3];
+  int32_t off_src;         // fp8 cache only, else 0: int32[n_desc] pool row (relative to the reservation) behind
+                           // every descriptor; the attention descriptors then carry staging rows instead
+  int32_t pad[2];
 };
 static_assert(sizeof(PlanHeader) % 16 == 0, "header must keep 16-byte alignment");
 
@@ -57,6 +59,8 @@ struct Plan {
   int layout = 0;
   int64_t reserved_rows = 0;            // multiple of HEATKV_PAGE_TOKENS
   int64_t peak_tokens = 0;
+  int64_t stage_rows = 0;               // fp8 cache: staging rows one attention call needs per sequence (64 per
+                                        // visible half-tile of the busiest (step, layer))
   std::vector<int32_t> blob;            // PlanHeader followed by the tables
   // host-only bookkeeping for introspection -------------------------------------------------
   // place[(l*H+h)*K + i] = first relative row of source scale i in the paged layout (-1: never stored)
@@ -93,6 +97,9 @@ SplitChoice split_search(const std::vector<int>& tiles, int n_qp, int n_seq, int
 
 int build_schedule(const heatkv_config& cfg, const double* scas, const double* cas, int policy,
                    int accounting, double b, const double* fraction, Schedule* out);
-int build_plan(const Schedule& sch, int layout, Plan* out);
+// `fp8`: plan for a context with the fp8 cache (paged layout only): the attention descriptors of every
+// (step, layer) are renumbered to consecutive 64-row staging slots, in descriptor order across the layer's heads,
+// and a table of the pool rows behind them is added.
+int build_plan(const Schedule& sch, int layout, Plan* out, bool fp8 = false);
 
 }  // namespace heatkv

@@ -23,6 +23,7 @@ struct Builder {
   std::vector<Move> moves;
   std::vector<int32_t> attn_begin, attn_cnt, app_begin, app_cnt, order;
   std::vector<int32_t> pre_begin, pre_cnt, post_begin, post_cnt;
+  std::vector<int32_t> src;                 // fp8 cache: pool row behind every descriptor
   explicit Builder(const Schedule& s) : S(s) {
     size_t n = (size_t)S.K * S.L * S.H;
     attn_begin.assign(n, 0); attn_cnt.assign(n, 0); app_begin.assign(n, 0); app_cnt.assign(n, 0);
@@ -59,6 +60,7 @@ struct Builder {
     h.off_pre_cnt = put(pre_cnt.data(), pre_cnt.size() * 4);
     h.off_post_begin = put(post_begin.data(), post_begin.size() * 4);
     h.off_post_cnt = put(post_cnt.data(), post_cnt.size() * 4);
+    if (!src.empty()) h.off_src = put(src.data(), src.size() * 4);
     while (b.size() % 4) b.push_back(0);
     h.total_words = (int32_t)b.size();
     *reinterpret_cast<PlanHeader*>(b.data()) = h;
@@ -88,8 +90,9 @@ void fill_order(const Schedule& S, Builder& B) {
 
 }  // namespace
 
-int build_plan(const Schedule& S, int layout, Plan* out) {
+int build_plan(const Schedule& S, int layout, Plan* out, bool fp8) {
   if (layout != HEATKV_LAYOUT_PAGED && layout != HEATKV_LAYOUT_RAGGED) return HEATKV_ERR_INVALID_ARG;
+  if (fp8 && layout != HEATKV_LAYOUT_PAGED) return HEATKV_ERR_INVALID_ARG;
   const int L = S.L, H = S.H, K = S.K, s = S.s, T = L * H;
   Builder B(S);
   fill_order(S, B);
@@ -286,6 +289,21 @@ int build_plan(const Schedule& S, int layout, Plan* out) {
     }
   }
   out->peak_tokens = peak_tokens;
+  out->stage_rows = 0;
+  if (fp8) {
+    // The attention kernels read bf16 staging rows that the call fills from the fp8 pool just before: the
+    // visible half-tiles of a (step, layer) take consecutive 64-row slots in descriptor order (the layer's
+    // heads are emitted one after the other), and `src` keeps the pool row of every descriptor.
+    B.src.resize(B.descs.size());
+    for (size_t i = 0; i < B.descs.size(); ++i) B.src[i] = B.descs[i].row;
+    for (int k = 0; k < K; ++k)
+      for (int l = 0; l < L; ++l) {
+        const int32_t first = B.attn_begin[S.at(k, l, 0)];
+        const int32_t end = B.attn_begin[S.at(k, l, H - 1)] + B.attn_cnt[S.at(k, l, H - 1)];
+        for (int32_t i = first; i < end; ++i) B.descs[i].row = (i - first) * P;
+        out->stage_rows = std::max<int64_t>(out->stage_rows, (int64_t)(end - first) * P);
+      }
+  }
   B.finish(out);
   return HEATKV_OK;
 }

@@ -22,12 +22,13 @@ __all__ = [
     "heatkv_finalize_scores", "heatkv_build_schedule", "heatkv_schedule_free", "heatkv_schedule_masks", "heatkv_schedule_footprint",
     "heatkv_schedule_plan", "heatkv_seq_open", "heatkv_seq_close", "heatkv_append_compact", "heatkv_scale_attention",
     "heatkv_attention_append", "heatkv_split_plan",
-    "heatkv_cache_bytes", "heatkv_retained_indices", "heatkv_export_head", "heatkv_allocator_stats",
-    "heatkv_launch_count", "heatkv_kernel_launches", "heatkv_rank_dispersion", "heatkv_seq_reservation", "KernelStats",
+    "heatkv_cache_bytes", "heatkv_retained_indices", "heatkv_export_head", "heatkv_export_head_fp8", "heatkv_allocator_stats",
+    "CACHE_BF16", "CACHE_FP8_E4M3", "heatkv_launch_count", "heatkv_kernel_launches", "heatkv_rank_dispersion", "heatkv_seq_reservation", "KernelStats",
     "heatkv_selftest_wait_expiry", "heatkv_device_status", "heatkv_strerror", "heatkv_attention_split", "arena_bytes_for",
 ]
 
 MAX_K, MAX_BATCH, PAGE_TOKENS = 16, 128, 64
+CACHE_BF16, CACHE_FP8_E4M3 = 0, 1
 LAYOUT_RAGGED, LAYOUT_PAGED = 0, 1
 POLICY_HEATKV, POLICY_BINARY, POLICY_NAIVE, POLICY_EXPLICIT = 0, 1, 2, 3
 ACCOUNT_PHYSICAL, ACCOUNT_LITERAL = 0, 1
@@ -44,18 +45,20 @@ class Config(C.Structure):
     _fields_ = [("L", C.c_int32), ("H", C.c_int32), ("d", C.c_int32), ("K", C.c_int32),
                 ("t", C.c_int32 * MAX_K), ("s", C.c_int32), ("layout", C.c_int32), ("kernel", C.c_int32),
                 ("sm_scale", C.c_float), ("arena", C.c_void_p), ("arena_bytes", C.c_uint64),
-                ("meta_bytes", C.c_uint64), ("scratch_bytes", C.c_uint64)]
+                ("meta_bytes", C.c_uint64), ("scratch_bytes", C.c_uint64),
+                ("cache_dtype", C.c_int32), ("reserved0", C.c_int32), ("stage_bytes", C.c_uint64)]
 
     @classmethod
     def make(cls, L: int, H: int, d: int, t: Sequence[int], s: int, layout: int = LAYOUT_PAGED,
              kernel: int = KERNEL_AUTO, sm_scale: float = 0.0, arena: Optional[torch.Tensor] = None,
-             meta_bytes: int = 0, scratch_bytes: int = 0) -> "Config":
+             meta_bytes: int = 0, scratch_bytes: int = 0, cache_dtype: int = 0, stage_bytes: int = 0) -> "Config":
         cfg = cls()
         cfg.L, cfg.H, cfg.d, cfg.K, cfg.s = L, H, d, len(t), s
         for i, v in enumerate(t):
             cfg.t[i] = int(v)
         cfg.layout, cfg.kernel, cfg.sm_scale, cfg.meta_bytes = layout, kernel, sm_scale, meta_bytes
         cfg.scratch_bytes = scratch_bytes
+        cfg.cache_dtype, cfg.stage_bytes = cache_dtype, stage_bytes
         if arena is not None:
             cfg.arena = arena.data_ptr()
             cfg.arena_bytes = arena.numel() * arena.element_size()
@@ -100,7 +103,7 @@ def exported_symbols():
             "heatkv_build_schedule", "heatkv_schedule_free", "heatkv_schedule_masks",
             "heatkv_schedule_footprint", "heatkv_schedule_plan", "heatkv_seq_open", "heatkv_seq_close", "heatkv_append_compact",
             "heatkv_scale_attention", "heatkv_attention_append", "heatkv_cache_bytes", "heatkv_seq_reservation",
-            "heatkv_retained_indices", "heatkv_export_head",
+            "heatkv_retained_indices", "heatkv_export_head", "heatkv_export_head_fp8",
             "heatkv_attention_split", "heatkv_split_plan", "heatkv_allocator_stats", "heatkv_launch_count",
             "heatkv_kernel_launches", "heatkv_rank_dispersion", "heatkv_selftest_wait_expiry", "heatkv_device_status",
             "heatkv_strerror"]
@@ -142,6 +145,7 @@ _lib.heatkv_attention_split.argtypes = [_P, C.POINTER(C.c_int), C.c_int, C.c_int
 _lib.heatkv_cache_bytes.argtypes = [_P, C.c_int, C.POINTER(C.c_uint64), C.POINTER(C.c_uint64)]
 _lib.heatkv_retained_indices.argtypes = [_P, C.c_int, C.c_int, C.c_int, _P, C.POINTER(C.c_int)]
 _lib.heatkv_export_head.argtypes = [_P, C.c_int, C.c_int, C.c_int, _P, _P, _P]
+_lib.heatkv_export_head_fp8.argtypes = [_P, C.c_int, C.c_int, C.c_int, _P, _P, _P, _P, _P]
 _lib.heatkv_allocator_stats.argtypes = [_P, C.POINTER(AllocStats)]
 _lib.heatkv_launch_count.argtypes = [_P, C.POINTER(C.c_uint64)]
 _lib.heatkv_device_status.argtypes = [_P, _P]
@@ -183,11 +187,15 @@ def heatkv_strerror(status: int) -> str:
     return _lib.heatkv_strerror(int(status)).decode()
 
 
-def arena_bytes_for(pool_rows: int, d: int, meta_bytes: int = 1 << 24, scratch_bytes: int = 1 << 26) -> int:
+def arena_bytes_for(pool_rows: int, d: int, meta_bytes: int = 1 << 24, scratch_bytes: int = 1 << 26,
+                    cache_dtype: int = 0, stage_bytes: int = 0) -> int:
     """Arena size that yields at least `pool_rows` rows in each of the K and V pools when the context is
-    created with the same (non-zero) `meta_bytes` and `scratch_bytes`."""
+    created with the same (non-zero) `meta_bytes`, `scratch_bytes` and, for the fp8 cache, `stage_bytes`."""
     rows = (pool_rows + PAGE_TOKENS - 1) // PAGE_TOKENS * PAGE_TOKENS
-    return (meta_bytes + 1023) // 1024 * 1024 + (scratch_bytes + 1023) // 1024 * 1024 + 2 * rows * d * 2
+    fixed = (meta_bytes + 1023) // 1024 * 1024 + (scratch_bytes + 1023) // 1024 * 1024
+    if cache_dtype == CACHE_FP8_E4M3:
+        return fixed + stage_bytes + 2 * rows * (d + 1)
+    return fixed + 2 * rows * d * 2
 
 
 def heatkv_create(cfg: Config, stream=None) -> int:
@@ -337,6 +345,11 @@ def heatkv_retained_indices(ctx: int, seq_id: int, layer: int, head: int, max_to
     n = C.c_int()
     _check(_lib.heatkv_retained_indices(ctx, seq_id, layer, head, _ptr(idx), C.byref(n)), "heatkv_retained_indices")
     return idx[: n.value].copy()
+
+
+def heatkv_export_head_fp8(ctx, seq_id, layer, head, k_codes, v_codes, k_exps, v_exps, stream=None) -> None:
+    _check(_lib.heatkv_export_head_fp8(ctx, seq_id, layer, head, _ptr(k_codes), _ptr(v_codes), _ptr(k_exps), _ptr(v_exps),
+                                       _stream(stream)), "heatkv_export_head_fp8")
 
 
 def heatkv_export_head(ctx, seq_id, layer, head, k_out, v_out, stream=None) -> None:

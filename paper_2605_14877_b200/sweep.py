@@ -15,17 +15,20 @@ class Session:
 
     def __init__(self, L: int, H: int, d: int, t: Sequence[int], s: int, pool_rows: int,
                  layout: int = hk.LAYOUT_PAGED, kernel: int = hk.KERNEL_AUTO, sm_scale: float = 0.0,
-                 meta_bytes: int = 1 << 24, device: str = "cuda:0", scratch_bytes: int = 1 << 26):
+                 meta_bytes: int = 1 << 24, device: str = "cuda:0", scratch_bytes: int = 1 << 26,
+                 cache_dtype: int = hk.CACHE_BF16, stage_bytes: int = 0):
         self.L, self.H, self.d, self.t, self.s = L, H, d, list(t), s
         self.K = len(self.t)
         self.c = [sum(self.t[: i + 1]) for i in range(self.K)]
         self.device = torch.device(device)
-        nbytes = hk.arena_bytes_for(pool_rows, d, meta_bytes, scratch_bytes)
+        if cache_dtype == hk.CACHE_FP8_E4M3 and stage_bytes == 0:
+            stage_bytes = 64 << 20                     # bf16 staging rows of one attention call (K and V)
+        nbytes = hk.arena_bytes_for(pool_rows, d, meta_bytes, scratch_bytes, cache_dtype, stage_bytes)
         self.arena = torch.empty(nbytes + 1024, dtype=torch.uint8, device=self.device)
         off = (-self.arena.data_ptr()) % 1024
         self._arena_view = self.arena[off: off + nbytes]
         self.cfg = hk.Config.make(L, H, d, self.t, s, layout, kernel, sm_scale, self._arena_view, meta_bytes,
-                                  scratch_bytes)
+                                  scratch_bytes, cache_dtype, stage_bytes)
         self.ctx = hk.heatkv_create(self.cfg)
 
     def close(self) -> None:
