@@ -258,11 +258,12 @@ def run_reference(args, rank):
     print(json.dumps(line), flush=True)
 
 
-def cache_update_numbers(reps, cases=("append_paged", "append_ragged", "compact_ragged"), first_scale=1):
+def cache_update_numbers(reps, cases=("append_paged", "append_ragged", "compact_ragged", "append_fp8_paged"), first_scale=1):
     """Cache-update kernels at a saturating shape: the larger-model layer shape (32 heads, d=128, 16 sequences,
     one layer).  Appends are timed with every head storing (full budget, paged and ragged); the in-place
     compaction of the ragged layout under a 1/5 budget.  Bytes are algorithmic: 8*d*t_k per storing head (K and
-    V, read + write), 8*d*moved tokens per move.  Rows for scales >= first_scale."""
+    V, read + write), 8*d*moved tokens per move; the quantising append of the fp8 cache reads 4*d and writes 2*(d+1) bytes per
+    token.  Rows for scales >= first_scale."""
     import paper_2605_14877_b200 as hk
     from paper_2605_14877_b200.sweep import Session
     sh = W.Shape("larger_layer", L=1, H=32, d=128, sides=W.SIDES_13, n_seq=16, s=3)
@@ -274,10 +275,12 @@ def cache_update_numbers(reps, cases=("append_paged", "append_ragged", "compact_
     flush = torch.empty(256 << 20, dtype=torch.uint8, device="cuda")
     stream = torch.cuda.current_stream()
     for name, layout, b in (("append_paged", hk.LAYOUT_PAGED, 1.0), ("append_ragged", hk.LAYOUT_RAGGED, 1.0),
-                            ("compact_ragged", hk.LAYOUT_RAGGED, 0.2)):
+                            ("compact_ragged", hk.LAYOUT_RAGGED, 0.2), ("append_fp8_paged", hk.LAYOUT_PAGED, 1.0)):
         if name not in cases:
             continue
-        ses = Session(sh.L, sh.H, sh.d, sh.t, sh.s, pool_rows=sh.n_seq * sh.H * (sh.c[-2] + 64 * sh.K) + 64, layout=layout)
+        fp8 = name == "append_fp8_paged"
+        ses = Session(sh.L, sh.H, sh.d, sh.t, sh.s, pool_rows=sh.n_seq * sh.H * (sh.c[-2] + 64 * sh.K) + 64, layout=layout,
+                      cache_dtype=hk.CACHE_FP8_E4M3 if fp8 else hk.CACHE_BF16)
         sch = ses.schedule(scas=W.synthetic_scas(sh, 0), b=b)
         am, km, nk, _ = hk.heatkv_schedule_masks(sch, sh.K, sh.L, sh.H)
         plan = hk.heatkv_schedule_plan(sch, layout)
@@ -306,6 +309,8 @@ def cache_update_numbers(reps, cases=("append_paged", "append_ragged", "compact_
         for step in range(first_scale - 1, sh.K - 1):
             storing = sum(1 for h in range(sh.H) if (int(km[step, 0, h]) >> step) & 1)
             nbytes = 8 * sh.d * sh.t[step] * storing * sh.n_seq
+            if fp8:      # K and V: 2 d bytes read, d codes + 1 exponent byte written, per token
+                nbytes = 2 * (2 * sh.d + sh.d + 1) * sh.t[step] * storing * sh.n_seq
             if name == "compact_ragged":
                 # plus the tokens moved by both evictions of the step: the plan's move lists (src, dst, n, 0)
                 off_move = int(hdr[10])
@@ -423,6 +428,53 @@ def run_head_dim_64_workload(args):
         res[name + "_ms_per_scale"] = [round(float(x), 4) for x in ms]
         res[name + "_sum_ms"] = round(float(ms.sum()), 4)
         res[name + "_tflops_largest"] = round(flops[sh.K - 1] / (float(ms[sh.K - 1]) * 1e-3) / 1e12, 1)
+        hk.heatkv_schedule_free(sch)
+        ses.close()
+    print(json.dumps(res), flush=True)
+
+
+def run_fp8_cache_workload(args):
+    """The single-layer workload (16 heads, d=128, 13 scales, batch 2, budget 1/20) with the bf16 cache and with
+    the fp8 cache (not the headline line): layer sweeps timed call by call, heatkv_attention_append per step.
+    With the fp8 cache a step is three kernels (expansion of the visible rows, attention, quantising append)
+    instead of one; the cache at the end of the sweep takes (d + 1) / (2 d) of the bytes."""
+    import paper_2605_14877_b200 as hk
+    from paper_2605_14877_b200.sweep import Session
+    torch.cuda.set_device(0)
+    sh = W.CFG2
+    scores = W.synthetic_scas(sh, 0)
+    q, k, v = W.qkv_layer(sh, 0, 0, device="cuda")
+    c = [0] + sh.c
+    qs, ks, vs = ([x[:, :, c[i]:c[i + 1]].contiguous() for i in range(sh.K)] for x in (q, k, v))
+    outs = [torch.zeros_like(x) for x in qs]
+    flush = torch.empty(256 << 20, dtype=torch.uint8, device="cuda")
+    res = {"workload": "fp8_cache_single_layer", "H": sh.H, "d": sh.d, "n_seq": sh.n_seq, "budget": B_BUDGET,
+           "scores": "synthetic"}
+    for name, dtype in (("bf16", hk.CACHE_BF16), ("fp8", hk.CACHE_FP8_E4M3)):
+        ses = Session(sh.L, sh.H, sh.d, sh.t, sh.s, pool_rows=2 * sh.n_seq * sh.H * (sh.c[-2] + 64 * sh.K), cache_dtype=dtype)
+        sch = ses.schedule(scas=scores, b=B_BUDGET)
+        ms, reps = np.zeros(sh.K), max(3, min(args.steps, 20))
+        n0 = hk.heatkv_launch_count(ses.ctx)
+        for rep in range(reps + 2):
+            ids = [hk.heatkv_seq_open(ses.ctx, sch) for _ in range(sh.n_seq)]
+            for step in range(sh.K):
+                ses.pre_step(ids, step)
+                flush.fill_(1)
+                e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+                e0.record()
+                hk.heatkv_attention_append(ses.ctx, ids, 0, step, qs[step], ks[step], vs[step], None, None, outs[step])
+                e1.record()
+                torch.cuda.synchronize()
+                if rep >= 2:
+                    ms[step] += e0.elapsed_time(e1) / reps
+            if rep == reps + 1:
+                res[name + "_cache_bytes_per_sequence"] = int(hk.heatkv_cache_bytes(ses.ctx, ids[0])[0])
+            for i in ids:
+                hk.heatkv_seq_close(ses.ctx, i)
+        assert hk.heatkv_device_status(ses.ctx) == 0
+        res[name + "_ms_per_scale"] = [round(float(x), 4) for x in ms]
+        res[name + "_sum_ms"] = round(float(ms.sum()), 4)
+        res[name + "_launches_per_sweep"] = int((hk.heatkv_launch_count(ses.ctx) - n0) // (reps + 2))
         hk.heatkv_schedule_free(sch)
         ses.close()
     print(json.dumps(res), flush=True)
@@ -592,7 +644,7 @@ def main():
     ap.add_argument("--calls", default="fused", choices=["fused", "separate"],
                     help="fused: heatkv_attention_append (one launch per step in the paged layout); separate: "
                          "heatkv_scale_attention followed by heatkv_append_compact")
-    ap.add_argument("--workload", default="config2", choices=["config2", "cache", "full", "larger", "serving", "fewheads", "stability", "d64"],
+    ap.add_argument("--workload", default="config2", choices=["config2", "cache", "full", "larger", "serving", "fewheads", "stability", "d64", "fp8"],
                     help="config2: the headline line; cache: append / compaction GB/s at a saturating shape; "
                          "full / larger / serving: whole-model sweeps of the other workloads; fewheads: key-range "
                          "splitting on launches with few (sequence, head) units; stability: S-CAS rank spread "
@@ -622,6 +674,10 @@ def main():
         return
     if args.workload == "d64":
         run_head_dim_64_workload(args)
+        return
+    if args.workload == "fp8":
+        if rank == 0:
+            run_fp8_cache_workload(args)
         return
     if args.workload == "fewheads":
         if rank == 0:
@@ -855,11 +911,12 @@ def main():
                 if per_step_kernels["attention_tcgen05"] else "attn_generic_kernel<%d> (mma.sync)" % shape.d)
     cache_update = None
     if rank == 0 and world == 1 and args.layout == "paged":
-        cu = cache_update_numbers(5, cases=("append_paged", "compact_ragged"), first_scale=9)
+        cu = cache_update_numbers(5, cases=("append_paged", "compact_ragged", "append_fp8_paged"), first_scale=9)
         cache_update = {"shape": cu["shape"], "peak_gbs": cu["peak_gbs"], "peak_source": cu["peak_source"],
                         "append_kernel_paged": cu["append_paged"], "append_plus_compact_kernel_ragged_budget_1_5": cu["compact_ragged"],
+                        "append_fp8_kernel_paged": cu["append_fp8_paged"],
                         "kernels_launched": {"append_paged": cu["append_paged_kernels"], "compact_ragged": cu["compact_ragged_kernels"]},
-                        "bytes": "algorithmic: 8*d*t_k per storing head, 8*d per moved token"}
+                        "bytes": "algorithmic: 8*d*t_k per storing head, 8*d per moved token; fp8 append: (4*d + 2*(d+1))*t_k per storing head"}
 
     # ---- roofline of the dominant kernel, all its launches of a layer sweep
     pk = peaks()
