@@ -235,6 +235,12 @@ int heatkv_schedule_footprint(const heatkv_schedule* sch, int layout, int64_t* p
  * the per-(step, layer, head) tables are indexed (step*L + layer)*H + head.
  * Call with words == NULL to get *n_words, then with a buffer of that many int32.        */
 int heatkv_schedule_plan(const heatkv_schedule* sch, int layout, int32_t* words, int64_t* n_words);
+/* The same for a context with the fp8 cache (paged layout): the attention descriptors of every (step, layer) carry
+ * staging rows -- consecutive 64-row slots in descriptor order across the layer's heads -- and header word 17 is the
+ * word offset of an extra table int32[n_desc] with the pool row behind every descriptor (append descriptors keep
+ * pool rows).  *stage_rows (optional) = staging rows one sequence needs in an attention call: 64 per visible
+ * half-tile of its busiest (step, layer).  Pure host code. */
+int heatkv_schedule_plan_fp8(const heatkv_schedule* sch, int32_t* words, int64_t* n_words, int64_t* stage_rows);
 
 /* Admit / retire one image.  Opening reserves the sequence's rows for its whole life (the
  * schedule is static, so the reservation and every page table are known up front) and, on

@@ -568,6 +568,25 @@ int heatkv_schedule_plan(const heatkv_schedule* sch, int layout, int32_t* words,
   return HEATKV_OK;
 }
 
+int heatkv_schedule_plan_fp8(const heatkv_schedule* sch, int32_t* words, int64_t* n_words, int64_t* stage_rows) {
+  if (!sch || !n_words) return HEATKV_ERR_INVALID_ARG;
+  Plan plan;
+  int rc;
+  try {
+    rc = build_plan(sch->s, HEATKV_LAYOUT_PAGED, &plan, true);
+  } catch (const std::bad_alloc&) {
+    return HEATKV_ERR_HOST_MEMORY;
+  }
+  if (rc != HEATKV_OK) return rc;
+  if (words) {
+    if (*n_words < (int64_t)plan.blob.size()) return HEATKV_ERR_INVALID_ARG;
+    std::memcpy(words, plan.blob.data(), plan.blob.size() * 4);
+  }
+  *n_words = (int64_t)plan.blob.size();
+  if (stage_rows) *stage_rows = plan.stage_rows;
+  return HEATKV_OK;
+}
+
 int heatkv_seq_open(heatkv_ctx* ctx, const heatkv_schedule* sch, void* stream_, int* seq_id) {
   if (!ctx || !sch || !seq_id) return HEATKV_ERR_INVALID_ARG;
   cudaStream_t stream = static_cast<cudaStream_t>(stream_);

@@ -20,7 +20,7 @@ __all__ = [
     "MAX_K", "MAX_BATCH", "PAGE_TOKENS",
     "heatkv_create", "heatkv_destroy", "heatkv_calibrate_scores", "heatkv_calibrate_scores_static",
     "heatkv_finalize_scores", "heatkv_build_schedule", "heatkv_schedule_free", "heatkv_schedule_masks", "heatkv_schedule_footprint",
-    "heatkv_schedule_plan", "heatkv_seq_open", "heatkv_seq_close", "heatkv_append_compact", "heatkv_scale_attention",
+    "heatkv_schedule_plan", "heatkv_schedule_plan_fp8", "heatkv_seq_open", "heatkv_seq_close", "heatkv_append_compact", "heatkv_scale_attention",
     "heatkv_attention_append", "heatkv_split_plan",
     "heatkv_cache_bytes", "heatkv_retained_indices", "heatkv_export_head", "heatkv_export_head_fp8", "heatkv_allocator_stats",
     "CACHE_BF16", "CACHE_FP8_E4M3", "heatkv_launch_count", "heatkv_kernel_launches", "heatkv_rank_dispersion", "heatkv_seq_reservation", "KernelStats",
@@ -101,7 +101,7 @@ def exported_symbols():
     return ["heatkv_create", "heatkv_destroy", "heatkv_calibrate_scores", "heatkv_calibrate_scores_static",
             "heatkv_finalize_scores",
             "heatkv_build_schedule", "heatkv_schedule_free", "heatkv_schedule_masks",
-            "heatkv_schedule_footprint", "heatkv_schedule_plan", "heatkv_seq_open", "heatkv_seq_close", "heatkv_append_compact",
+            "heatkv_schedule_footprint", "heatkv_schedule_plan", "heatkv_schedule_plan_fp8", "heatkv_seq_open", "heatkv_seq_close", "heatkv_append_compact",
             "heatkv_scale_attention", "heatkv_attention_append", "heatkv_cache_bytes", "heatkv_seq_reservation",
             "heatkv_retained_indices", "heatkv_export_head", "heatkv_export_head_fp8",
             "heatkv_attention_split", "heatkv_split_plan", "heatkv_allocator_stats", "heatkv_launch_count",
@@ -131,6 +131,7 @@ _lib.heatkv_schedule_free.argtypes = [_P]
 _lib.heatkv_schedule_masks.argtypes = [_P, _P, _P, _P, C.POINTER(C.c_int64)]
 _lib.heatkv_schedule_footprint.argtypes = [_P, C.c_int, C.POINTER(C.c_int64), C.POINTER(C.c_int64)]
 _lib.heatkv_schedule_plan.argtypes = [_P, C.c_int, _P, C.POINTER(C.c_int64)]
+_lib.heatkv_schedule_plan_fp8.argtypes = [_P, _P, C.POINTER(C.c_int64), C.POINTER(C.c_int64)]
 _lib.heatkv_seq_open.argtypes = [_P, _P, _P, C.POINTER(C.c_int)]
 _lib.heatkv_seq_close.argtypes = [_P, C.c_int]
 _lib.heatkv_append_compact.argtypes = [_P, C.POINTER(C.c_int), C.c_int, C.c_int, C.c_int, _P, _P, C.POINTER(Strides), _P]
@@ -271,6 +272,15 @@ def heatkv_schedule_plan(sch: int, layout: int) -> np.ndarray:
     words = np.zeros(n.value, dtype=np.int32)
     _check(_lib.heatkv_schedule_plan(sch, layout, _ptr(words), C.byref(n)), "heatkv_schedule_plan")
     return words
+
+
+def heatkv_schedule_plan_fp8(sch: int):
+    """(plan tables of a context with the fp8 cache as one int32 array, staging rows a sequence needs per call)."""
+    n, rows = C.c_int64(0), C.c_int64(0)
+    _check(_lib.heatkv_schedule_plan_fp8(sch, None, C.byref(n), None), "heatkv_schedule_plan_fp8")
+    words = np.zeros(n.value, dtype=np.int32)
+    _check(_lib.heatkv_schedule_plan_fp8(sch, _ptr(words), C.byref(n), C.byref(rows)), "heatkv_schedule_plan_fp8")
+    return words, rows.value
 
 
 def heatkv_seq_open(ctx: int, sch: int, stream=None) -> int:

@@ -379,3 +379,43 @@ def test_split_plan_rejects_bad_input():
         hk.heatkv_split_plan([3, 5], n_qp=1, n_seq=1)       # not in dispatch (descending) order
     with pytest.raises(hk.HeatKVError):
         hk.heatkv_split_plan([4, 0], n_qp=1, n_seq=1)
+
+
+def test_fp8_plan_renumbers_attention_rows_into_staging_slots(hk):
+    """Plan of a context with the fp8 cache against the plain paged plan of the same schedule: same tables, the
+    attention descriptors of every (step, layer) sit in consecutive 64-row staging slots in descriptor order, the
+    extra table holds the pool rows the plain plan has in their place, append descriptors keep their pool rows,
+    and the staging rows asked for are 64 per visible half-tile of the busiest (step, layer)."""
+    sh = W.Shape("mid", L=3, H=4, d=128, sides=W.SIDES_13[:11], n_seq=1, s=3)
+    cfg = hk.Config.make(sh.L, sh.H, sh.d, sh.t, sh.s)
+    sch = hk.heatkv_build_schedule(cfg, scas=W.synthetic_scas(sh, 4), b=0.15)
+    plain = hk.heatkv_schedule_plan(sch, hk.LAYOUT_PAGED)
+    fp8, stage_rows = hk.heatkv_schedule_plan_fp8(sch)
+    hk.heatkv_schedule_free(sch)
+    n_desc = int(plain[3])
+    assert int(fp8[3]) == n_desc and int(plain[17]) == 0 and int(fp8[17]) > 0
+    for w in range(4, 15):                               # every table of the plain plan sits at the same offset
+        assert int(plain[w]) == int(fp8[w])
+    pd = plain[int(plain[4]): int(plain[4]) + 2 * n_desc].reshape(n_desc, 2)
+    fd = fp8[int(fp8[4]): int(fp8[4]) + 2 * n_desc].reshape(n_desc, 2)
+    src = fp8[int(fp8[17]): int(fp8[17]) + n_desc]
+    assert np.array_equal(pd[:, 1], fd[:, 1])            # valid rows and source scales unchanged
+    assert np.array_equal(src, pd[:, 0])                 # the pool rows moved into the extra table
+    n_units = sh.K * sh.L * sh.H
+    ab, ac = plain[int(plain[5]): int(plain[5]) + n_units], plain[int(plain[6]): int(plain[6]) + n_units]
+    pb, pc = plain[int(plain[7]): int(plain[7]) + n_units], plain[int(plain[8]): int(plain[8]) + n_units]
+    is_attn = np.zeros(n_desc, dtype=bool)
+    busiest = 0
+    for k in range(sh.K):
+        for l in range(sh.L):
+            u0 = (k * sh.L + l) * sh.H
+            first, end = int(ab[u0]), int(ab[u0 + sh.H - 1] + ac[u0 + sh.H - 1])
+            for h in range(sh.H):                        # the layer's heads follow one another without gaps
+                assert int(ab[u0 + h]) == first + int(ac[u0: u0 + h].sum())
+            assert np.array_equal(fd[first:end, 0], 64 * np.arange(end - first))
+            is_attn[first:end] = True
+            busiest = max(busiest, end - first)
+    for u in range(n_units):                             # append descriptors keep pool rows
+        b0, n = int(pb[u]), int(pc[u])
+        assert not is_attn[b0: b0 + n].any() and np.array_equal(fd[b0: b0 + n, 0], pd[b0: b0 + n, 0])
+    assert stage_rows == 64 * busiest and busiest > 0
