@@ -161,3 +161,13 @@ def test_fp8_cache_needs_paged_layout_and_enough_staging(hk):
             ses.generate(ids, lambda l: (q, k, v), lambda l: out)
         assert ei.value.status == -4                      # HEATKV_ERR_OUT_OF_PAGES
         hk.heatkv_schedule_free(sch)
+
+
+def test_fp8_cache_config2_full_size(hk):
+    """Config 2 (16 heads, d=128, 13 scales, batch 2, 20x) with the fp8 cache at full size, automatic kernel
+    choice, one call per (layer, step): every (sequence, head) unit against the oracle."""
+    sh = W.CFG2
+    scores = W.synthetic_scas(sh, 0)
+    ref = O.heatkv_schedule(scores, 0.05, sh.s, sh.sides)
+    bias = W.seg_bias_current_scale(sh, 0)
+    _run_fp8(hk, sh, ref, lambda ses: ses.schedule(scas=scores, b=0.05), hk.KERNEL_AUTO, bias=bias, fused=True)
