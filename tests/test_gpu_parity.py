@@ -469,6 +469,43 @@ def test_config2_calibration_full_size(hk):
         assert np.isclose(cas[0, h], O.cas(ref, sh.s), rtol=RTOL_BETA, atol=1e-9)
 
 
+def test_config3_calibration_sixteen_samples(hk):
+    """Calibration as config 3 runs it, on one layer of its shape: 16 seeded samples (two calls of 8 sequences per
+    step, accumulated in the same beta), per-head log-normal bias on the prior scales, automatic kernel choice.
+    beta and S-CAS of three heads over all 16 samples against the oracle at 1e-3 relative; unit row sums and an empty
+    upper triangle for every head."""
+    from paper_2605_14877_b200.sweep import Session
+    sh = W.Shape("cfg3_layer", L=1, H=16, d=128, sides=W.SIDES_13, n_seq=8, s=3)
+    sm = 1.0 / math.sqrt(sh.d)
+    bias = W.seg_bias_prior_lognormal(sh, 0)
+    bias_dev = torch.from_numpy(bias).cuda()
+    beta_dev = torch.zeros(sh.L, sh.H, sh.K, sh.K, dtype=torch.float32, device="cuda")
+    heads, batches = (1, 6, 12), 2
+    ref = {h: np.zeros((sh.K, sh.K)) for h in heads}
+    with Session(sh.L, sh.H, sh.d, sh.t, sh.s, pool_rows=64, kernel=hk.KERNEL_AUTO) as ses:
+        for bt in range(batches):
+            q, k, _ = W.qkv_layer(sh, 200 + bt, 0, device="cuda")
+            for step in range(sh.K):
+                lo, hi = ses.step_slices(step)
+                qs, ks_ = q[:, :, lo:hi], k[:, :, :hi]
+                hk.heatkv_calibrate_scores(ses.ctx, 0, step, sh.n_seq, qs, ks_, None, hk.Strides.of(qs, ks_),
+                                           bias_dev[0, step], beta_dev, None)
+            for head in heads:
+                qh, kh = _f64(q[:, head]), _f64(k[:, head])
+                for s_ in range(sh.n_seq):
+                    ref[head] += O.beta_sample(qh[s_], kh[s_], sh.sides, sm, bias[0, :, head, :].astype(np.float64))
+        beta, scas, _ = hk.heatkv_finalize_scores(ses.ctx, beta_dev, batches * sh.n_seq, sh.L, sh.H, sh.K)
+        assert hk.heatkv_device_status(ses.ctx) == 0
+    assert np.allclose(beta.sum(axis=-1), 1.0, atol=2e-4)
+    assert np.all(np.triu(beta, 1) == 0)
+    for head in heads:
+        want = ref[head] / (batches * sh.n_seq)
+        mask = want > 1e-5
+        rel = np.abs(beta[0, head] - want)[mask] / want[mask]
+        assert rel.max() <= RTOL_BETA, (head, float(rel.max()))
+        assert np.allclose(scas[0, head], O.scas(want, sh.s), rtol=RTOL_BETA, atol=1e-9)
+
+
 def test_calibration_without_output_ignores_output_strides(hk):
     """A C caller that computes no attention output may leave the o_* strides zero (both calibration entry
     points); the result is the one the call with filled-in strides gives."""
