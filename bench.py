@@ -522,7 +522,11 @@ def run_stability_workload(args):
 
 
 def run_model_workload(args, which):
-    """Whole-model sweeps (not the headline line).  `full`: 2B-class full model cache, 32 layers x 16
+    print(json.dumps(model_workload(which, max(1, min(args.steps, 3)), args.launch == "graph")), flush=True)
+
+
+def model_workload(which, reps, with_graph, only_budget=None):
+    """Whole-model sweeps (not the headline metric).  `full`: 2B-class full model cache, 32 layers x 16
     heads, batch 8, budgets 1/5, 1/10, 1/20.  `larger`: 40 layers x 32 heads, batch 16, 1/20.  `serving`:
     64 concurrent images of the 2B shape, per-request budgets from {1/5, 1/10, 1/20, 1/40}, paged cache,
     four admission waves one scale apart.  All layers reuse one layer's seeded activations (the kernels see
@@ -538,8 +542,8 @@ def run_model_workload(args, which):
     out = torch.zeros_like(data[0])
     cfg0 = hk.Config.make(sh.L, sh.H, sh.d, sh.t, sh.s)
     results = []
-    runs = {"full": [[b] * sh.n_seq for b in (1 / 5, 1 / 10, 1 / 20)], "larger": [[1 / 20] * sh.n_seq],
-            "serving": [W.serving_budgets(sh.n_seq, 0)]}[which]
+    runs = {"full": [[b] * sh.n_seq for b in (1 / 5, 1 / 10, 1 / 20) if only_budget is None or abs(b - only_budget) < 1e-9],
+            "larger": [[1 / 20] * sh.n_seq], "serving": [W.serving_budgets(sh.n_seq, 0)]}[which]
     n_waves = 4 if which == "serving" else 1
     wave = sh.n_seq // n_waves
     for budgets in runs:
@@ -581,7 +585,6 @@ def run_model_workload(args, which):
 
         generation(False)
         torch.cuda.synchronize()
-        reps = max(1, min(args.steps, 3))
         e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
         t0 = time.perf_counter()
         e0.record(stream)
@@ -593,7 +596,7 @@ def run_model_workload(args, which):
         assert hk.heatkv_device_status(ses.ctx) == 0
         # the same generation as one CUDA graph (all launches of all layers and scales), replayed
         graph_ms = None
-        if args.launch == "graph":
+        if with_graph:
             side = torch.cuda.Stream()
             side.wait_stream(torch.cuda.current_stream())
             with torch.cuda.stream(side):
@@ -613,11 +616,19 @@ def run_model_workload(args, which):
             graph_ms = e0.elapsed_time(e1) / reps
             assert hk.heatkv_device_status(ses.ctx) == 0
         n_images = sh.n_seq / (2 if which != "serving" else 1)      # cond/uncond pair = one image outside serving
+        # algorithmic attention flops of the generation (4*d*t_k*n_vis over all sequences, layers, heads, scales)
+        gen_flops = 0
+        for b in sorted(set(budgets)):
+            am_b = hk.heatkv_schedule_masks(schs[b], sh.K, sh.L, sh.H)[0]
+            gen_flops += sum(attention_flops(sh, am_b, sum(1 for x in budgets if x == b)))
+        best_ms = min(ms, graph_ms) if graph_ms is not None else ms
         full_bytes = sh.n_seq * sh.L * sh.H * sh.c[-2] * sh.d * 4
         results.append({"budgets": sorted(set(round(b, 4) for b in budgets)), "ms_per_generation": round(ms, 2),
                         "images_per_s": round(n_images / (ms * 1e-3), 2),
                         "graph_ms_per_generation": None if graph_ms is None else round(graph_ms, 2),
                         "graph_images_per_s": None if graph_ms is None else round(n_images / (graph_ms * 1e-3), 2),
+                        "attention_tflops": round(gen_flops / (best_ms * 1e-3) / 1e12, 1),
+                        "attention_frac_of_bf16_peak": round(gen_flops / (best_ms * 1e-3) / 1e12 / peaks()["bf16_tflops_sustained"], 3),
                         "cache_GB_end": round(a.used_tokens * sh.d * 4 / 1e9, 3),
                         "cache_GB_uncompressed": round(full_bytes / 1e9, 3),
                         "reserved_GB": round(a.reserved_rows * sh.d * 4 / 1e9, 3),
@@ -626,8 +637,12 @@ def run_model_workload(args, which):
         for sch in schs.values():
             hk.heatkv_schedule_free(sch)
         ses.close()
-    print(json.dumps({"workload": sh.name, "L": sh.L, "H": sh.H, "n_seq": sh.n_seq, "launch": "calls issued from Python (ms_per_generation) and one CUDA graph replay (graph_*)",
-                      "data": "synthetic, one layer's activations reused by all layers", "runs": results}), flush=True)
+    del data, out
+    torch.cuda.empty_cache()
+    return ({"workload": sh.name, "L": sh.L, "H": sh.H, "n_seq": sh.n_seq, "launch": "calls issued from Python (ms_per_generation) and one CUDA graph replay (graph_*)",
+                      "data": "synthetic, one layer's activations reused by all layers",
+                      "peak": "attention_frac_of_bf16_peak is against the %s sustained bf16 figure (a generation lasts tens of milliseconds and more)" % peaks()["source"],
+                      "runs": results})
 
 
 def main():
@@ -975,6 +990,12 @@ def main():
         line["cache_update"] = cache_update
     hk.heatkv_schedule_free(sch)
     ses.close()
+    if rank == 0 and world == 1 and args.layout == "paged" and args.kernel == "auto" and N_LAYERS == 32:
+        # the same model at the batch the paper's full-model workload has (8 sequences = 4 image pairs, 32 layers,
+        # budget 1/20): launches large enough to fill the GPU; fraction against the sustained bf16 peak
+        del layer_bufs, flush
+        torch.cuda.empty_cache()
+        line["full_model_batch8"] = model_workload("full", 2, True, only_budget=B_BUDGET)
     if dist is not None:
         dist.barrier()
         dist.destroy_process_group()
