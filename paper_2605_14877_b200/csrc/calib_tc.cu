@@ -7,14 +7,19 @@
 //
 // One CTA owns 256 queries of one (sequence, head) as two 128-row tiles A and B.  Warp roles:
 //   warp 0      TMA producer: Q tiles once, then K half-tiles (64 rows x 128 dims) of the full key set,
-//               cut at source-scale borders (descriptor list built on the host), 4 stages.
+//               cut at source-scale borders (descriptor list built on the host), 3 stages.
 //   warp 1      MMA issuer: S_x = Q_x K^T into TMEM as soon as the softmax warps have read the
 //               previous S_x into registers (they say so right after the load, before the exponentials).
-//   warps 4-7   tile A, warps 8-11 tile B: one thread per query row keeps the running max, the row sum
-//               and the mass of the scale it is inside; finished scales are parked in shared memory
-//               relative to the same reference and rescaled when the reference moves (rare).
-// At the end every row's masses are divided by its row sum, summed over the CTA's rows and added to
-// beta with one atomicAdd per (CTA, source scale).  Every wait is bounded as in the attention kernel.
+//   warps 4-11  tile A, warps 12-19 tile B: TWO threads per query row, one for keys 0..63 and one for keys
+//               64..127 of every key tile (warps w and w + 4 share a TMEM lane quadrant).  Nothing here needs
+//               a reference common to a row while the tiles stream by (there is no P to hand to a product),
+//               so each thread keeps a running max, a sum and the mass of the scale it is inside of its own --
+//               a half-tile lies inside one source scale -- parks finished scales in shared memory relative to
+//               its own reference and rescales them when that moves (rare).  Four softmax warps per SM
+//               sub-partition instead of two keep the exponential unit fed.
+// At the end the two halves of every row are brought to a common reference, the row's masses are divided by
+// its row sum, summed over the CTA's rows and added to beta with one atomicAdd per (CTA, source scale).  Every
+// wait is bounded as in the attention kernel.
 #include <new>
 #include <vector>
 
@@ -27,29 +32,33 @@ namespace calib {
 
 using namespace tc;
 
-constexpr int D_MAX = 128;               // the shared-memory map is sized for 128-wide heads; 64-wide ones use half of each tile
+// (the shared-memory map is sized for 128-wide heads; 64-wide ones use half of each tile)
 constexpr int BM = 128;                 // rows per Q tile
 constexpr int BN = 128;                 // keys per tile (two 64-row half-tiles)
 constexpr int HALF = 64;
-constexpr int THREADS = 384;
-constexpr int K_STAGES = 4;
+constexpr int THREADS = 640;             // 4 utility warps + 16 softmax warps
+constexpr int REGS_UTIL = 40, REGS_SOFTMAX = 104, REGS_LAUNCH = 96;   // ptxas assigns 96 under __launch_bounds__(640, 1)
+static_assert(128 * REGS_UTIL + 512 * REGS_SOFTMAX <= THREADS * REGS_LAUNCH, "register hand-over exceeds the CTA's allocation");
+constexpr int K_STAGES = 3;               // with the per-thread scale masses of two threads per row, four would not fit
 constexpr uint32_t HALF_COLS_BYTES = 128 * 128;        // one 64-column half of a 128-row tile: 16 KB
 constexpr uint32_t TILE_BYTES = 2 * HALF_COLS_BYTES;   // 32 KB
 constexpr uint32_t SLOT_BYTES = HALF * 128;            // 64 rows x 128 B inside one column half
 
 constexpr uint32_t SM_Q = 0;                                   // 2 tiles
 constexpr uint32_t SM_K = SM_Q + 2 * TILE_BYTES;               // K_STAGES tiles
-constexpr uint32_t SM_SEG = SM_K + K_STAGES * TILE_BYTES;      // float[2 tiles][16 scales][128 rows]
-constexpr uint32_t SM_ACC = SM_SEG + 2 * HEATKV_MAX_K * BM * 4;  // float[16]: the CTA's sums per scale
+constexpr uint32_t SM_SEG = SM_K + K_STAGES * TILE_BYTES;      // float[2 tiles][2 key halves][16 scales][128 rows]
+constexpr uint32_t SM_STAT = SM_SEG + 4 * HEATKV_MAX_K * BM * 4;  // float[2 tiles][2 key halves][2][128 rows]: reference, sum
+constexpr uint32_t SM_ACC = SM_STAT + 4 * 2 * BM * 4;          // float[16]: the CTA's sums per scale
 constexpr uint32_t SM_BAR = SM_ACC + HEATKV_MAX_K * 4;
 constexpr uint32_t SM_TOTAL = SM_BAR + 256;
 constexpr uint32_t SM_ALLOC = SM_TOTAL + 1024;                 // slack for manual alignment
+static_assert(SM_ALLOC <= 227 * 1024, "shared memory of one CTA");
 
 enum Bar : uint32_t {
   Q_FULL = 0,                   // +x (2)
-  K_FULL = 2, K_EMPTY = 6,      // +stage (4 each)
+  K_FULL = 2, K_EMPTY = 6,      // +stage (K_STAGES each, room for 4)
   S_FULL = 10,                  // +x  S_x of tile j is in TMEM
-  S_READ = 12,                  // +x  the 128 rows of S_x of tile j are in registers (128 arrivals)
+  S_READ = 12,                  // +x  the 128 rows of S_x of tile j are in registers (256 arrivals: two threads per row)
   N_BARS = 14
 };
 constexpr uint32_t SM_TMEM_PTR = SM_BAR + N_BARS * 8;
@@ -104,7 +113,7 @@ calib_tc_kernel(const __grid_constant__ AttnParams p, const __grid_constant__ Ma
     for (int x = 0; x < 2; ++x) {
       mbar_init(bar(Q_FULL + x), 1);
       mbar_init(bar(S_FULL + x), 1);
-      mbar_init(bar(S_READ + x), BM);
+      mbar_init(bar(S_READ + x), 2 * BM);
     }
     for (int s = 0; s < K_STAGES; ++s) {
       mbar_init(bar(K_FULL + s), 1);
@@ -124,14 +133,14 @@ calib_tc_kernel(const __grid_constant__ AttnParams p, const __grid_constant__ Ma
   tc_fence_after();
   const uint32_t tmem = *tmem_ptr_smem;
 
-  // register budget per warpgroup: 128*72 + 256*216 <= 384*168
+  // register budget per warpgroup: 128*40 + 512*104 <= 640*96
   if (warp < 4) {
-    reg_dealloc<72>();
+    reg_dealloc<REGS_UTIL>();
     if (warp == 0) {
       // ------------------------------------------------------------------ TMA producer
       const bool leader = elect_one();
       uint32_t armed = 0;                               // stage -> a copy was issued at least once
-      uint32_t par[K_STAGES] = {0, 0, 0, 0};
+      uint32_t par[K_STAGES] = {};
       if (leader) {
         for (int x = 0; x < nq; ++x) {
           mbar_expect_tx(bar(Q_FULL + x), LOAD_BYTES);
@@ -196,65 +205,55 @@ calib_tc_kernel(const __grid_constant__ AttnParams p, const __grid_constant__ Ma
       }
     }
   } else {
-    reg_alloc<216>();
+    reg_alloc<REGS_SOFTMAX>();
     // ------------------------------------------------------------------ softmax with per-scale masses
-    const int x = (warp - 4) >> 2;                      // 0: tile A, 1: tile B
+    const int x = (warp - 4) >> 3;                      // 0: tile A (warps 4-11), 1: tile B (warps 12-19)
+    const int g = ((warp - 4) >> 2) & 1;                // which 64 keys of every key tile
+    const int row = (warp & 3) * 32 + lane;             // row inside the tile == TMEM lane
+    float* seg_smem = reinterpret_cast<float*>(sgen + SM_SEG) + (x * 2 + g) * (HEATKV_MAX_K * BM);   // [scale][row]
+    float* stat_smem = reinterpret_cast<float*>(sgen + SM_STAT) + (x * 2 + g) * (2 * BM);           // [reference | sum][row]
+    float m_ref = -INFINITY, l_sum = 0.f;
+    int cur_seg = -1;                                   // the scale whose mass is being collected (warp-uniform)
+    float cur_sum = 0.f;
+    bool ok = true;
     if (x < nq) {
-      const int row = (warp & 3) * 32 + lane;           // row inside the tile == TMEM lane
-      const uint32_t t_s = tmem + ((uint32_t)((warp & 3) * 32) << 16) + x * 128;
-      float* seg_smem = reinterpret_cast<float*>(sgen + SM_SEG) + x * (HEATKV_MAX_K * BM);   // [scale][row]
+      const uint32_t t_s = tmem + ((uint32_t)((warp & 3) * 32) << 16) + x * 128 + g * 64;
       const float* bias_h = p.seg_bias ? p.seg_bias + head * p.K : nullptr;
       const float LOG2E = 1.4426950408889634f;
-      float m_ref = -INFINITY, l_sum = 0.f;
-      int cur_seg = -1;                                 // the scale whose mass is being collected (warp-uniform)
-      float cur_sum = 0.f;
-      bool ok = true;
       for (int j = 0; j < n_tiles && ok; ++j) {
-        const HalfTile s0 = get_half(2 * j, descs, n_slots), s1 = get_half(2 * j + 1, descs, n_slots);
-        const float b0 = bias_h ? bias_h[s0.seg] * LOG2E : 0.f;
-        const float b1 = bias_h ? bias_h[s1.seg] * LOG2E : 0.f;
+        const HalfTile sg = get_half(2 * j + g, descs, n_slots);
+        const float bg = bias_h ? bias_h[sg.seg] * LOG2E : 0.f;
         ok = __all_sync(0xffffffffu, mbar_wait(bar(S_FULL + x), j & 1, abort_flag, p.status));
         if (!ok) break;
         tc_fence_after();
-        uint32_t r0[32], r1[32], r2[32], r3[32];
+        uint32_t r0[32], r1[32];
         tmem_ld32(t_s, r0);
         tmem_ld32(t_s + 32, r1);
-        tmem_ld32(t_s + 64, r2);
-        tmem_ld32(t_s + 96, r3);
         tmem_wait_ld();
         tc_fence_before();
         mbar_arrive(bar(S_READ + x));                   // the next S_x may overwrite these columns
-        if (s0.n_valid < HALF || s1.n_valid < HALF) {   // ragged tile (warp-uniform): mask by -inf
+        if (sg.n_valid == 0) continue;                  // padding half-tile (warp-uniform): nothing to add
+        if (sg.n_valid < HALF) {                        // ragged half-tile (warp-uniform): mask by -inf
 #pragma unroll
           for (int i = 0; i < 32; ++i) {
-            if (i >= s0.n_valid) r0[i] = 0xff800000u;
-            if (i + 32 >= s0.n_valid) r1[i] = 0xff800000u;
-            if (i >= s1.n_valid) r2[i] = 0xff800000u;
-            if (i + 32 >= s1.n_valid) r3[i] = 0xff800000u;
+            if (i >= sg.n_valid) r0[i] = 0xff800000u;
+            if (i + 32 >= sg.n_valid) r1[i] = 0xff800000u;
           }
         }
-        // row maximum: the logit is raw * scale + bias(half) with scale > 0, so take the raw maxima
-        float mq[8];
+        // maximum of the 64 logits: the logit is raw * scale + bias(half) with scale > 0, so take the raw maximum
+        float mq[4];
 #pragma unroll
-        for (int c = 0; c < 4; ++c) {
-          mq[c] = fmaxf(__uint_as_float(r0[c]), __uint_as_float(r1[c]));
-          mq[4 + c] = fmaxf(__uint_as_float(r2[c]), __uint_as_float(r3[c]));
-        }
+        for (int c = 0; c < 4; ++c) mq[c] = fmaxf(__uint_as_float(r0[c]), __uint_as_float(r1[c]));
 #pragma unroll
         for (int i = 4; i < 32; i += 4) {
 #pragma unroll
-          for (int c = 0; c < 4; ++c) {
-            mq[c] = fmax3(mq[c], __uint_as_float(r0[i + c]), __uint_as_float(r1[i + c]));
-            mq[4 + c] = fmax3(mq[4 + c], __uint_as_float(r2[i + c]), __uint_as_float(r3[i + c]));
-          }
+          for (int c = 0; c < 4; ++c) mq[c] = fmax3(mq[c], __uint_as_float(r0[i + c]), __uint_as_float(r1[i + c]));
         }
-        const float mx0 = fmaxf(fmaxf(mq[0], mq[1]), fmaxf(mq[2], mq[3]));
-        const float mx1 = fmaxf(fmaxf(mq[4], mq[5]), fmaxf(mq[6], mq[7]));
-        const float mx = fmaxf(fmaf(mx0, p.scale_log2, b0), fmaf(mx1, p.scale_log2, b1));
+        const float mx = fmaf(fmaxf(fmaxf(mq[0], mq[1]), fmaxf(mq[2], mq[3])), p.scale_log2, bg);
         const float m_new = fmaxf(m_ref, mx);
         const bool grow = m_new > m_ref + RESCALE_THRESHOLD;   // also true on the first tile (m_ref = -inf)
         if (grow) {
-          if (j > 0) {
+          if (m_ref > -INFINITY) {
             // everything collected so far is relative to m_ref: move it to the new reference
             const float f = exp2f(m_ref - m_new);
             l_sum *= f;
@@ -265,10 +264,12 @@ calib_tc_kernel(const __grid_constant__ AttnParams p, const __grid_constant__ Ma
         }
         __syncwarp();
         const uint64_t scale2 = pack2(p.scale_log2, p.scale_log2);
-        auto exp_sum = [&](const uint32_t (&rc)[32], uint64_t bb2, uint64_t& sum2) {
+        const uint64_t bb = pack2(bg - m_ref, bg - m_ref);
+        uint64_t sum_a = pack2(0.f, 0.f), sum_b = pack2(0.f, 0.f);
+        auto exp_sum = [&](const uint32_t (&rc)[32], uint64_t& sum2) {
 #pragma unroll
           for (int i = 0; i < 32; i += 2) {
-            const uint64_t xx = fma2(pack2(__uint_as_float(rc[i]), __uint_as_float(rc[i + 1])), scale2, bb2);
+            const uint64_t xx = fma2(pack2(__uint_as_float(rc[i]), __uint_as_float(rc[i + 1])), scale2, bb);
             float e0, e1;
             if (((i >> 1) % 3) == 2) {                  // one pair in three on the FMA pipe (measured best for this kernel)
               exp2_poly2(xx, e0, e1);
@@ -281,44 +282,56 @@ calib_tc_kernel(const __grid_constant__ AttnParams p, const __grid_constant__ Ma
             sum2 = add2(sum2, pack2(e0, e1));
           }
         };
-        const uint64_t bb0 = pack2(b0 - m_ref, b0 - m_ref), bb1 = pack2(b1 - m_ref, b1 - m_ref);
-        uint64_t sum_h0 = pack2(0.f, 0.f), sum_h1 = pack2(0.f, 0.f);
-        exp_sum(r0, bb0, sum_h0);
-        exp_sum(r1, bb0, sum_h0);
-        exp_sum(r2, bb1, sum_h1);
-        exp_sum(r3, bb1, sum_h1);
+        exp_sum(r0, sum_a);
+        exp_sum(r1, sum_b);
         float a0, a1, c0, c1;
-        unpack2(sum_h0, a0, a1);
-        unpack2(sum_h1, c0, c1);
-        const float h0 = a0 + a1, h1 = c0 + c1;
-        l_sum += h0 + h1;
+        unpack2(sum_a, a0, a1);
+        unpack2(sum_b, c0, c1);
+        const float h = (a0 + a1) + (c0 + c1);
+        l_sum += h;
         // source scales arrive in ascending order, each as one run of half-tiles
-        if (s0.seg != cur_seg) {
+        if (sg.seg != cur_seg) {
           if (cur_seg >= 0) seg_smem[cur_seg * BM + row] = cur_sum;
-          cur_seg = s0.seg;
+          // scales this thread never sees between the two (their half-tiles all went to the partner) stay zero
+          for (int s = cur_seg + 1; s < sg.seg; ++s) seg_smem[s * BM + row] = 0.f;
+          cur_seg = sg.seg;
           cur_sum = 0.f;
         }
-        cur_sum += h0;
-        if (s1.n_valid > 0) {
-          if (s1.seg != cur_seg) {
-            seg_smem[cur_seg * BM + row] = cur_sum;
-            cur_seg = s1.seg;
-            cur_sum = 0.f;
-          }
-          cur_sum += h1;
-        }
+        cur_sum += h;
       }
       if (ok) {
-        seg_smem[cur_seg * BM + row] = cur_sum;
-        // Eq. 2: mean over the step's rows of mass(row, scale) / rowsum(row); rows past t_q are padding
-        const bool live = q0 + x * BM + row < p.t_q;
-        const float inv = live ? 1.f / l_sum : 0.f;
-        for (int s = 0; s <= p.step; ++s) {
-          float v = live ? seg_smem[s * BM + row] * inv : 0.f;
+        if (cur_seg >= 0) seg_smem[cur_seg * BM + row] = cur_sum;
+        for (int s = cur_seg + 1; s <= p.step; ++s) seg_smem[s * BM + row] = 0.f;
+        stat_smem[row] = m_ref;
+        stat_smem[BM + row] = l_sum;
+      }
+    }
+  }
+
+  // ---- the two halves of every row meet: thread (row, keys 0..63) brings both to a common reference
+  tc_fence_before();
+  __syncthreads();
+  if (warp >= 4 && ((warp - 4) >> 2 & 1) == 0 && *abort_flag == 0) {
+    const int x = (warp - 4) >> 3;
+    if (x < nq) {
+      const int row = (warp & 3) * 32 + lane;
+      const float* seg0 = reinterpret_cast<const float*>(sgen + SM_SEG) + (x * 2) * (HEATKV_MAX_K * BM);
+      const float* seg1 = seg0 + HEATKV_MAX_K * BM;
+      const float* st0 = reinterpret_cast<const float*>(sgen + SM_STAT) + (x * 2) * (2 * BM);
+      const float* st1 = st0 + 2 * BM;
+      // Eq. 2: mean over the step's rows of mass(row, scale) / rowsum(row); rows past t_q are padding.  A thread
+      // that saw no valid key keeps the reference -inf and contributes nothing.
+      const float m0 = st0[row], m1 = st1[row];
+      const float m = fmaxf(m0, m1);
+      const float w0 = m0 > -INFINITY ? exp2f(m0 - m) : 0.f, w1 = m1 > -INFINITY ? exp2f(m1 - m) : 0.f;
+      const float l = st0[BM + row] * w0 + st1[BM + row] * w1;
+      const bool live = q0 + x * BM + row < p.t_q;
+      const float inv = live ? 1.f / l : 0.f;
+      for (int s = 0; s <= p.step; ++s) {
+        float v = live ? (seg0[s * BM + row] * w0 + seg1[s * BM + row] * w1) * inv : 0.f;
 #pragma unroll
-          for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
-          if (lane == 0) atomicAdd(acc_smem + s, v);
-        }
+        for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
+        if (lane == 0) atomicAdd(acc_smem + s, v);
       }
     }
   }
@@ -401,7 +414,7 @@ int calib_tc_create(const heatkv_config& cfg, void* dev_table, cudaStream_t stre
     return HEATKV_OK;
   }
   // the register hand-over inside the kernel must fit in what the launch really allocates
-  if (attr.numRegs * calib::THREADS < 128 * 72 + 256 * 216) return HEATKV_ERR_CUDA;
+  if (attr.numRegs * calib::THREADS < 128 * calib::REGS_UTIL + 512 * calib::REGS_SOFTMAX) return HEATKV_ERR_CUDA;
   st->ready = true;
   return HEATKV_OK;
 }
