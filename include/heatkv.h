@@ -171,6 +171,21 @@ int heatkv_calibrate_scores(heatkv_ctx* ctx, int layer, int step, int n_seq, con
                             const void* k_full, const void* v_full, const heatkv_strides* st,
                             const float* seg_bias, float* beta_accum, void* out, void* stream);
 
+/* Sec. 3.1, Eq. 2 for the steps step_begin .. step_end - 1 of one layer in one call: offline calibration from
+ * recorded activations, where the queries and keys of every scale of a sample are at hand (the beta rows of different
+ * steps are independent of one another).  The steps the tensor-memory kernel takes run as ONE launch whose CTAs are
+ * dispatched longest first, which evens out the rounds that a launch per step leaves partly filled; the small steps run
+ * on the generic kernel, one launch each.  Results agree with step-by-step heatkv_calibrate_scores calls up to the
+ * order of the fp32 sums.
+ *   q_all   DEVICE bf16 [n_seq,H,c[step_end-1],d]  the queries of all scales, token axis = the scales one after the
+ *           other, strides q_*
+ *   k_all   DEVICE bf16 [n_seq,H,c[step_end-1],d]  the keys, same layout, strides kv_*
+ *   seg_bias DEVICE fp32 [step_end][H][K]: the bias of step k at seg_bias + k*H*K, or NULL
+ *   beta_accum as in heatkv_calibrate_scores.  The o_* strides are not read. */
+int heatkv_calibrate_scores_steps(heatkv_ctx* ctx, int layer, int step_begin, int step_end, int n_seq, const void* q_all,
+                                  const void* k_all, const heatkv_strides* st, const float* seg_bias, float* beta_accum,
+                                  void* stream);
+
 /* No counterpart in the paper: heatkv_calibrate_scores for callers that must not allocate device
  * memory while they run -- code inside a serving loop whose memory pool is fixed at start-up, a plug-in
  * of a host application that owns the allocator, a caller between stream-ordered allocator

@@ -34,6 +34,9 @@ void calib_tc_destroy(CalibTcState* st);
 bool calib_tc_ready(const CalibTcState* st);
 bool calib_tc_supported(const CalibTcState* st, const AttnParams& p, int d, int n_seq);
 cudaError_t launch_calib_tc(CalibTcState* st, const AttnParams& p, int n_seq, cudaStream_t stream);
+cudaError_t launch_calib_tc_steps(CalibTcState* st, const AttnParams& p, int n_seq, const int* steps, const int* t_q,
+                                  const int* q_tok0, int n_steps, int q_tokens, int k_tokens, int64_t bias_step_stride,
+                                  cudaStream_t stream);
 }  // namespace heatkv
 
 using namespace heatkv;
@@ -802,6 +805,66 @@ int heatkv_calibrate_scores(heatkv_ctx* ctx, int layer, int step, int n_seq, con
   ctx->launches += 1;
   (use_tc ? ctx->kstats.calibration_tcgen05 : ctx->kstats.calibration_generic) += 1;
   return e == cudaSuccess ? HEATKV_OK : HEATKV_ERR_CUDA;
+}
+
+int heatkv_calibrate_scores_steps(heatkv_ctx* ctx, int layer, int step_begin, int step_end, int n_seq, const void* q_all,
+                                  const void* k_all, const heatkv_strides* st, const float* seg_bias, float* beta_accum,
+                                  void* stream_) {
+  if (!ctx || !q_all || !k_all || !beta_accum) return HEATKV_ERR_INVALID_ARG;
+  if (!aligned16(q_all) || !aligned16(k_all)) return HEATKV_ERR_INVALID_ARG;
+  if (layer < 0 || layer >= ctx->cfg.L || step_begin < 0 || step_begin >= step_end || step_end > ctx->cfg.K || n_seq < 1 ||
+      n_seq > 65535)
+    return HEATKV_ERR_INVALID_ARG;
+  cudaStream_t stream = static_cast<cudaStream_t>(stream_);
+  const int64_t d = ctx->cfg.d, H = ctx->cfg.H, K = ctx->cfg.K, tokens = ctx->c[step_end - 1];
+  AttnParams p;
+  std::memset(&p, 0, sizeof(p));
+  heatkv_strides s;
+  if (!st) {   // dense: [n_seq, H, tokens, d]
+    s.q_tok = s.kv_tok = s.o_tok = d;
+    s.q_head = s.kv_head = s.o_head = d * tokens;
+    s.q_seq = s.kv_seq = s.o_seq = d * tokens * H;
+  } else {
+    int rc = check_strides(ctx, st, (int)tokens, &s, false);
+    if (rc != HEATKV_OK) return rc;
+  }
+  fill_common(ctx, &p, s);
+  p.layer = layer;
+  float* beta_layer = beta_accum + (int64_t)layer * H * K * K;
+  // the steps the tensor-memory kernel takes, as one launch
+  int big[HEATKV_MAX_K], big_t[HEATKV_MAX_K], big_tok0[HEATKV_MAX_K], n_big = 0;
+  const int choice = ctx->cfg.kernel;
+  p.q = static_cast<const __nv_bfloat16*>(q_all);
+  p.k_new = static_cast<const __nv_bfloat16*>(k_all);
+  const bool tc_ok = choice != HEATKV_KERNEL_GENERIC && calib_tc_supported(ctx->calib_tc, p, ctx->cfg.d, n_seq);
+  for (int k = step_begin; k < step_end; ++k) {
+    const bool use_tc = tc_ok && !(choice == HEATKV_KERNEL_AUTO && ctx->cfg.t[k] < 256);
+    if (use_tc) {
+      big[n_big] = k; big_t[n_big] = ctx->cfg.t[k]; big_tok0[n_big] = ctx->c[k] - ctx->cfg.t[k];
+      ++n_big;
+      continue;
+    }
+    AttnParams g = p;                                   // a small step: the generic kernel on the step's views
+    g.q = p.q + (int64_t)(ctx->c[k] - ctx->cfg.t[k]) * s.q_tok;
+    g.seg_bias = seg_bias ? seg_bias + (int64_t)k * H * K : nullptr;
+    g.t_q = ctx->cfg.t[k];
+    g.n_own = ctx->c[k];
+    g.step = k;
+    g.beta_row = beta_layer + (int64_t)k * K;
+    if (launch_attn_generic(g, ctx->cfg.d, n_seq, true, stream) != cudaSuccess) return HEATKV_ERR_CUDA;
+    ctx->launches += 1;
+    ctx->kstats.calibration_generic += 1;
+  }
+  if (n_big > 0) {
+    p.seg_bias = seg_bias;
+    p.beta_row = beta_layer;
+    if (launch_calib_tc_steps(ctx->calib_tc, p, n_seq, big, big_t, big_tok0, n_big, (int)tokens, (int)tokens,
+                              seg_bias ? H * K : 0, stream) != cudaSuccess)
+      return HEATKV_ERR_CUDA;
+    ctx->launches += 1;
+    ctx->kstats.calibration_tcgen05 += 1;
+  }
+  return HEATKV_OK;
 }
 
 int heatkv_calibrate_scores_static(heatkv_ctx* ctx, int layer, int step, int n_seq, const void* q, const void* k_full,

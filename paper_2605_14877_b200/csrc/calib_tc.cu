@@ -20,6 +20,8 @@
 // At the end the two halves of every row are brought to a common reference, the row's masses are divided by
 // its row sum, summed over the CTA's rows and added to beta with one atomicAdd per (CTA, source scale).  Every
 // wait is bounded as in the attention kernel.
+#include <algorithm>
+#include <cstring>
 #include <new>
 #include <vector>
 
@@ -69,6 +71,19 @@ struct Maps {
   CUtensorMap q, k;
 };
 
+// The steps one launch covers (one for heatkv_calibrate_scores, several for heatkv_calibrate_scores_steps): CTAs
+// cta_begin[e] .. cta_begin[e + 1] - 1 belong to entry e, query tile pair fastest, then sequence, then head.
+// Entries are ordered by descending work, so the long CTAs are dispatched first.
+struct StepTable {
+  int n;
+  int cta_begin[HEATKV_MAX_K + 1];
+  int step[HEATKV_MAX_K];
+  int t_q[HEATKV_MAX_K];        // queries of the step
+  int q_tok0[HEATKV_MAX_K];     // first query token of the step on the token axis of the q map
+  int desc_first[HEATKV_MAX_K]; // the step's key half-tiles in the descriptor table
+  int n_slots[HEATKV_MAX_K];
+};
+
 struct HalfTile {
   int row;          // first key row inside k_full
   int n_valid;      // real rows of the 64
@@ -87,8 +102,8 @@ __device__ __forceinline__ HalfTile get_half(int i, const int2* descs, int n_slo
 
 template <int D>
 __global__ void __launch_bounds__(THREADS, 1)
-calib_tc_kernel(const __grid_constant__ AttnParams p, const __grid_constant__ Maps maps, const int2* __restrict__ descs,
-                int n_slots) {
+calib_tc_kernel(const __grid_constant__ AttnParams p, const __grid_constant__ Maps maps, const int2* __restrict__ all_descs,
+                const __grid_constant__ StepTable tab, int n_seq, int64_t bias_step_stride) {
   static_assert(D == 64 || D == 128, "head dimension");
   constexpr int NCH = D / 64;                               // 64-column halves per row
   constexpr uint32_t LOAD_BYTES = NCH * HALF_COLS_BYTES;    // bytes one tile's copies deliver
@@ -102,9 +117,16 @@ calib_tc_kernel(const __grid_constant__ AttnParams p, const __grid_constant__ Ma
   auto bar = [&](uint32_t which) { return sbase + SM_BAR + which * 8; };
 
   const int warp = __shfl_sync(0xffffffffu, (int)(threadIdx.x >> 5), 0), lane = threadIdx.x & 31;
-  const int seq = blockIdx.y, head = blockIdx.z;
-  const int q0 = blockIdx.x * (2 * BM);
-  const int nq = (q0 + BM < p.t_q) ? 2 : 1;          // does tile B hold any query?
+  int e = 0;
+  while (e + 1 < tab.n && (int)blockIdx.x >= tab.cta_begin[e + 1]) ++e;
+  const int step = tab.step[e], t_q = tab.t_q[e], n_slots = tab.n_slots[e];
+  const int2* descs = all_descs + tab.desc_first[e];
+  const int n_qp = (t_q + 2 * BM - 1) / (2 * BM);
+  const int local = (int)blockIdx.x - tab.cta_begin[e];
+  const int seq = (local / n_qp) % n_seq, head = local / (n_qp * n_seq);
+  const int q0 = (local % n_qp) * (2 * BM);             // first query of the CTA inside its step
+  const int q_tok = tab.q_tok0[e] + q0;                 // ... and on the token axis of the q map
+  const int nq = (q0 + BM < t_q) ? 2 : 1;               // does tile B hold any query?
   const int n_tiles = (n_slots + 1) / 2;
 
   if (threadIdx.x == 0) {
@@ -147,7 +169,7 @@ calib_tc_kernel(const __grid_constant__ AttnParams p, const __grid_constant__ Ma
           for (int ch = 0; ch < NCH; ++ch)
             for (int hf = 0; hf < 2; ++hf)
               tma_load_4d(sbase + SM_Q + x * TILE_BYTES + ch * HALF_COLS_BYTES + hf * SLOT_BYTES, &maps.q, ch * 64,
-                          q0 + x * BM + hf * HALF, head, seq, bar(Q_FULL + x));
+                          q_tok + x * BM + hf * HALF, head, seq, bar(Q_FULL + x));
         }
       }
       bool ok = true;
@@ -218,7 +240,7 @@ calib_tc_kernel(const __grid_constant__ AttnParams p, const __grid_constant__ Ma
     bool ok = true;
     if (x < nq) {
       const uint32_t t_s = tmem + ((uint32_t)((warp & 3) * 32) << 16) + x * 128 + g * 64;
-      const float* bias_h = p.seg_bias ? p.seg_bias + head * p.K : nullptr;
+      const float* bias_h = p.seg_bias ? p.seg_bias + step * bias_step_stride + head * p.K : nullptr;
       const float LOG2E = 1.4426950408889634f;
       for (int j = 0; j < n_tiles && ok; ++j) {
         const HalfTile sg = get_half(2 * j + g, descs, n_slots);
@@ -301,7 +323,7 @@ calib_tc_kernel(const __grid_constant__ AttnParams p, const __grid_constant__ Ma
       }
       if (ok) {
         if (cur_seg >= 0) seg_smem[cur_seg * BM + row] = cur_sum;
-        for (int s = cur_seg + 1; s <= p.step; ++s) seg_smem[s * BM + row] = 0.f;
+        for (int s = cur_seg + 1; s <= step; ++s) seg_smem[s * BM + row] = 0.f;
         stat_smem[row] = m_ref;
         stat_smem[BM + row] = l_sum;
       }
@@ -325,9 +347,9 @@ calib_tc_kernel(const __grid_constant__ AttnParams p, const __grid_constant__ Ma
       const float m = fmaxf(m0, m1);
       const float w0 = m0 > -INFINITY ? exp2f(m0 - m) : 0.f, w1 = m1 > -INFINITY ? exp2f(m1 - m) : 0.f;
       const float l = st0[BM + row] * w0 + st1[BM + row] * w1;
-      const bool live = q0 + x * BM + row < p.t_q;
+      const bool live = q0 + x * BM + row < t_q;
       const float inv = live ? 1.f / l : 0.f;
-      for (int s = 0; s <= p.step; ++s) {
+      for (int s = 0; s <= step; ++s) {
         float v = live ? (seg0[s * BM + row] * w0 + seg1[s * BM + row] * w1) * inv : 0.f;
 #pragma unroll
         for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
@@ -338,8 +360,9 @@ calib_tc_kernel(const __grid_constant__ AttnParams p, const __grid_constant__ Ma
 
   tc_fence_before();
   __syncthreads();
-  if ((int)threadIdx.x <= p.step && *abort_flag == 0)
-    atomicAdd(p.beta_row + (int64_t)head * p.K * p.K + threadIdx.x, acc_smem[threadIdx.x] / (float)p.t_q);
+  // p.beta_row is beta_accum[layer][0][0]: the row of (head, step) follows
+  if ((int)threadIdx.x <= step && *abort_flag == 0)
+    atomicAdd(p.beta_row + ((int64_t)head * p.K + step) * p.K + threadIdx.x, acc_smem[threadIdx.x] / (float)t_q);
   if (warp == 0) {
     tc_fence_after();
     asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem), "r"(TMEM_COLS) : "memory");
@@ -445,19 +468,52 @@ bool encode_4d(CalibTcState* st, CUtensorMap* m, const void* base, int t, int H,
 }
 }  // namespace
 
-cudaError_t launch_calib_tc(CalibTcState* st, const AttnParams& p, int n_seq, cudaStream_t stream) {
+// One launch for the given steps of one layer.  `p` carries the common fields: q = the queries at token 0 of the
+// q map (`q_tokens` tokens per head), k_new = the keys (`k_tokens` per head), strides, H, K, seg_bias (of step 0
+// when `bias_step_stride` != 0, else of the one step), beta_row = beta_accum[layer][0][0].  `q_tok0[i]` is the first
+// query token of steps[i] on the q map's token axis.
+cudaError_t launch_calib_tc_steps(CalibTcState* st, const AttnParams& p, int n_seq, const int* steps, const int* t_q,
+                                  const int* q_tok0, int n_steps, int q_tokens, int k_tokens, int64_t bias_step_stride,
+                                  cudaStream_t stream) {
+  if (n_steps < 1 || n_steps > HEATKV_MAX_K) return cudaErrorInvalidValue;
   calib::Maps maps;
-  if (!encode_4d(st, &maps.q, p.q, p.t_q, p.H, n_seq, p.q_tok, p.q_head, p.q_seq) ||
-      !encode_4d(st, &maps.k, p.k_new, p.n_own, p.H, n_seq, p.kv_tok, p.kv_head, p.kv_seq))
+  if (!encode_4d(st, &maps.q, p.q, q_tokens, p.H, n_seq, p.q_tok, p.q_head, p.q_seq) ||
+      !encode_4d(st, &maps.k, p.k_new, k_tokens, p.H, n_seq, p.kv_tok, p.kv_head, p.kv_seq))
     return cudaErrorInvalidValue;
-  dim3 grid((p.t_q + 2 * calib::BM - 1) / (2 * calib::BM), n_seq, p.H);
+  // longest CTAs first: entries by descending key half-tiles (the CTAs of one step are all alike)
+  int order[HEATKV_MAX_K];
+  for (int i = 0; i < n_steps; ++i) order[i] = i;
+  std::sort(order, order + n_steps, [&](int a, int b) { return st->count[steps[a]] > st->count[steps[b]]; });
+  calib::StepTable tab;
+  std::memset(&tab, 0, sizeof(tab));
+  tab.n = n_steps;
+  int ctas = 0;
+  for (int e = 0; e < n_steps; ++e) {
+    const int i = order[e];
+    tab.cta_begin[e] = ctas;
+    tab.step[e] = steps[i];
+    tab.t_q[e] = t_q[i];
+    tab.q_tok0[e] = q_tok0[i];
+    tab.desc_first[e] = st->first[steps[i]];
+    tab.n_slots[e] = st->count[steps[i]];
+    ctas += (t_q[i] + 2 * calib::BM - 1) / (2 * calib::BM) * n_seq * p.H;
+  }
+  tab.cta_begin[n_steps] = ctas;
+  dim3 grid((unsigned)ctas);
   if (st->d == 128)
-    calib::calib_tc_kernel<128><<<grid, calib::THREADS, calib::SM_ALLOC, stream>>>(p, maps, st->dev_descs + st->first[p.step],
-                                                                                   st->count[p.step]);
+    calib::calib_tc_kernel<128><<<grid, calib::THREADS, calib::SM_ALLOC, stream>>>(p, maps, st->dev_descs, tab, n_seq, bias_step_stride);
   else
-    calib::calib_tc_kernel<64><<<grid, calib::THREADS, calib::SM_ALLOC, stream>>>(p, maps, st->dev_descs + st->first[p.step],
-                                                                                  st->count[p.step]);
+    calib::calib_tc_kernel<64><<<grid, calib::THREADS, calib::SM_ALLOC, stream>>>(p, maps, st->dev_descs, tab, n_seq, bias_step_stride);
   return cudaGetLastError();
+}
+
+// One step: p.q = the step's queries, p.t_q of them; p.k_new = all p.n_own keys; p.beta_row = beta_accum[layer][0][step]
+// as the generic kernel takes it.
+cudaError_t launch_calib_tc(CalibTcState* st, const AttnParams& p, int n_seq, cudaStream_t stream) {
+  AttnParams q = p;
+  q.beta_row = p.beta_row - (int64_t)p.step * p.K;       // back to beta_accum[layer][0][0]
+  const int step = p.step, t_q = p.t_q, tok0 = 0;
+  return launch_calib_tc_steps(st, q, n_seq, &step, &t_q, &tok0, 1, p.t_q, p.n_own, 0, stream);
 }
 
 }  // namespace heatkv

@@ -18,7 +18,7 @@ __all__ = [
     "LAYOUT_RAGGED", "LAYOUT_PAGED", "POLICY_HEATKV", "POLICY_BINARY", "POLICY_NAIVE", "POLICY_EXPLICIT",
     "ACCOUNT_PHYSICAL", "ACCOUNT_LITERAL", "KERNEL_AUTO", "KERNEL_GENERIC", "KERNEL_TCGEN05",
     "MAX_K", "MAX_BATCH", "PAGE_TOKENS",
-    "heatkv_create", "heatkv_destroy", "heatkv_calibrate_scores", "heatkv_calibrate_scores_static",
+    "heatkv_create", "heatkv_destroy", "heatkv_calibrate_scores", "heatkv_calibrate_scores_steps", "heatkv_calibrate_scores_static",
     "heatkv_finalize_scores", "heatkv_build_schedule", "heatkv_schedule_free", "heatkv_schedule_masks", "heatkv_schedule_footprint",
     "heatkv_schedule_plan", "heatkv_schedule_plan_fp8", "heatkv_seq_open", "heatkv_seq_close", "heatkv_append_compact", "heatkv_scale_attention",
     "heatkv_attention_append", "heatkv_split_plan",
@@ -98,7 +98,7 @@ def lib_path() -> str:
 
 def exported_symbols():
     """Names declared in include/heatkv.h, in declaration order."""
-    return ["heatkv_create", "heatkv_destroy", "heatkv_calibrate_scores", "heatkv_calibrate_scores_static",
+    return ["heatkv_create", "heatkv_destroy", "heatkv_calibrate_scores", "heatkv_calibrate_scores_steps", "heatkv_calibrate_scores_static",
             "heatkv_finalize_scores",
             "heatkv_build_schedule", "heatkv_schedule_free", "heatkv_schedule_masks",
             "heatkv_schedule_footprint", "heatkv_schedule_plan", "heatkv_schedule_plan_fp8", "heatkv_seq_open", "heatkv_seq_close", "heatkv_append_compact",
@@ -125,6 +125,7 @@ _lib.heatkv_create.argtypes = [C.POINTER(Config), _P, C.POINTER(_P)]
 _lib.heatkv_destroy.argtypes = [_P]
 _lib.heatkv_calibrate_scores.argtypes = [_P, C.c_int, C.c_int, C.c_int, _P, _P, _P, C.POINTER(Strides), _P, _P, _P, _P]
 _lib.heatkv_calibrate_scores_static.argtypes = [_P, C.c_int, C.c_int, C.c_int, _P, _P, C.POINTER(Strides), _P, _P, _P]
+_lib.heatkv_calibrate_scores_steps.argtypes = [_P, C.c_int, C.c_int, C.c_int, C.c_int, _P, _P, C.POINTER(Strides), _P, _P, _P]
 _lib.heatkv_finalize_scores.argtypes = [_P, _P, C.c_int, _P, _P, _P, _P]
 _lib.heatkv_build_schedule.argtypes = [C.POINTER(Config), _P, _P, C.c_int, C.c_int, C.c_double, _P, C.POINTER(_P)]
 _lib.heatkv_schedule_free.argtypes = [_P]
@@ -215,6 +216,16 @@ def heatkv_calibrate_scores(ctx, layer, step, n_seq, q, k_full, v_full, strides,
     _check(_lib.heatkv_calibrate_scores(ctx, layer, step, n_seq, _ptr(q), _ptr(k_full), _ptr(v_full), st,
                                         _ptr(seg_bias), _ptr(beta_accum), _ptr(out), _stream(stream)),
            "heatkv_calibrate_scores")
+
+
+def heatkv_calibrate_scores_steps(ctx, layer, step_begin, step_end, n_seq, q_all, k_all, strides, seg_bias, beta_accum,
+                                  stream=None) -> None:
+    """Eq. 2 for steps step_begin .. step_end - 1 of one layer in one call (q_all, k_all: [n_seq, H, tokens, d] with
+    all scales on the token axis; seg_bias: [step_end, H, K] or None)."""
+    st = C.byref(strides) if strides is not None else None
+    _check(_lib.heatkv_calibrate_scores_steps(ctx, layer, step_begin, step_end, n_seq, _ptr(q_all), _ptr(k_all), st,
+                                              _ptr(seg_bias), _ptr(beta_accum), _stream(stream)),
+           "heatkv_calibrate_scores_steps")
 
 
 def heatkv_calibrate_scores_static(ctx, layer, step, n_seq, q, k_full, strides, seg_bias, beta_accum,

@@ -469,6 +469,61 @@ def test_config2_calibration_full_size(hk):
         assert np.isclose(cas[0, h], O.cas(ref, sh.s), rtol=RTOL_BETA, atol=1e-9)
 
 
+@pytest.mark.parametrize("with_bias", [False, True], ids=["plain", "bias"])
+def test_calibration_all_steps_in_one_call(hk, with_bias):
+    """heatkv_calibrate_scores_steps (Sec. 3.1, Eq. 2 for every step of a layer at once: one tensor-memory launch
+    over the large steps, longest CTAs first) at the config-2 shape: equal to step-by-step calls up to the order of
+    the fp32 sums, beta of two heads against the oracle, and a sub-range of steps on strided views."""
+    from paper_2605_14877_b200.sweep import Session
+    sh = W.CFG2
+    sm = 1.0 / math.sqrt(sh.d)
+    bias = W.seg_bias_current_scale(sh, 0)
+    bias_dev = torch.from_numpy(bias).cuda()                       # [L, K, H, K]
+    q, k, _ = W.qkv_layer(sh, 321, 0, device="cuda")
+    with Session(sh.L, sh.H, sh.d, sh.t, sh.s, pool_rows=64, kernel=hk.KERNEL_AUTO) as ses:
+        one = torch.zeros(sh.L, sh.H, sh.K, sh.K, dtype=torch.float32, device="cuda")
+        for step in range(sh.K):
+            lo, hi = ses.step_slices(step)
+            qs, ks_ = q[:, :, lo:hi], k[:, :, :hi]
+            hk.heatkv_calibrate_scores(ses.ctx, 0, step, sh.n_seq, qs, ks_, None, hk.Strides.of(qs, ks_),
+                                       bias_dev[0, step] if with_bias else None, one, None)
+        n0 = hk.heatkv_kernel_launches(ses.ctx)
+        allk = torch.zeros_like(one)
+        hk.heatkv_calibrate_scores_steps(ses.ctx, 0, 0, sh.K, sh.n_seq, q, k, hk.Strides.of(q, k),
+                                         bias_dev[0] if with_bias else None, allk)
+        n1 = hk.heatkv_kernel_launches(ses.ctx)
+        big = sum(1 for t in sh.t if t >= 256)
+        assert n1.calibration_tcgen05 - n0.calibration_tcgen05 == 1                       # one launch for the large steps
+        assert n1.calibration_generic - n0.calibration_generic == sh.K - big
+        # steps 8 .. 11 only, on views of a wider buffer (strides differ from the dense ones)
+        wide_q = torch.zeros(sh.n_seq, sh.H, sh.c[-1] + 8, sh.d, dtype=torch.bfloat16, device="cuda")
+        wide_k = torch.zeros_like(wide_q)
+        wide_q[:, :, : sh.c[-1]], wide_k[:, :, : sh.c[-1]] = q, k
+        part = torch.zeros_like(one)
+        vq, vk = wide_q[:, :, : sh.c[10]], wide_k[:, :, : sh.c[10]]
+        hk.heatkv_calibrate_scores_steps(ses.ctx, 0, 7, 11, sh.n_seq, vq, vk, hk.Strides.of(vq, vk),
+                                         bias_dev[0] if with_bias else None, part)
+        torch.cuda.synchronize()
+        assert hk.heatkv_device_status(ses.ctx) == 0
+        a, b, c = one.cpu().numpy()[0], allk.cpu().numpy()[0], part.cpu().numpy()[0]
+    mask = a > 1e-5
+    assert (np.abs(a - b)[mask] / a[mask]).max() <= 1e-4
+    assert np.all(b[~mask] <= 2e-5)
+    sel = np.zeros_like(mask)
+    sel[:, 7:11, :] = mask[:, 7:11, :]
+    assert (np.abs(a - c)[sel] / a[sel]).max() <= 1e-4
+    rest = np.ones_like(mask)
+    rest[:, 7:11, :] = False
+    assert np.all(c[rest] == 0)
+    qh, kh = _f64(q), _f64(k)
+    for h in (3, 12):
+        ref = np.zeros((sh.K, sh.K))
+        for s_ in range(sh.n_seq):
+            ref += O.beta_sample(qh[s_, h], kh[s_, h], sh.sides, sm, bias[0, :, h, :].astype(np.float64) if with_bias else None)
+        m = ref > 1e-5 * sh.n_seq
+        assert (np.abs(b[h] - ref)[m] / ref[m]).max() <= RTOL_BETA, h
+
+
 def test_config3_calibration_sixteen_samples(hk):
     """Calibration as config 3 runs it, on one layer of its shape: 16 seeded samples (two calls of 8 sequences per
     step, accumulated in the same beta), per-head log-normal bias on the prior scales, automatic kernel choice.
