@@ -245,7 +245,7 @@ calib_tc_kernel(const __grid_constant__ AttnParams p, const __grid_constant__ Ma
       for (int j = 0; j < n_tiles && ok; ++j) {
         const HalfTile sg = get_half(2 * j + g, descs, n_slots);
         const float bg = bias_h ? bias_h[sg.seg] * LOG2E : 0.f;
-        ok = __all_sync(0xffffffffu, mbar_wait(bar(S_FULL + x), j & 1, abort_flag, p.status));
+        ok = __all_sync(0xffffffffu, mbar_wait_hint(bar(S_FULL + x), j & 1, abort_flag, p.status));
         if (!ok) break;
         tc_fence_after();
         uint32_t r0[32], r1[32];
