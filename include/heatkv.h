@@ -174,8 +174,8 @@ int heatkv_calibrate_scores(heatkv_ctx* ctx, int layer, int step, int n_seq, con
 /* Sec. 3.1, Eq. 2 for the steps step_begin .. step_end - 1 of one layer in one call: offline calibration from
  * recorded activations, where the queries and keys of every scale of a sample are at hand (the beta rows of different
  * steps are independent of one another).  The steps the tensor-memory kernel takes run as ONE launch whose CTAs are
- * dispatched longest first, which evens out the rounds that a launch per step leaves partly filled; the small steps run
- * on the generic kernel, one launch each.  Results agree with step-by-step heatkv_calibrate_scores calls up to the
+ * dispatched longest first, which evens out the rounds that a launch per step leaves partly filled; the small steps
+ * share one launch of the generic kernel.  Results agree with step-by-step heatkv_calibrate_scores calls up to the
  * order of the fp32 sums.
  *   q_all   DEVICE bf16 [n_seq,H,c[step_end-1],d]  the queries of all scales, token axis = the scales one after the
  *           other, strides q_*

@@ -837,20 +837,24 @@ int heatkv_calibrate_scores_steps(heatkv_ctx* ctx, int layer, int step_begin, in
   p.q = static_cast<const __nv_bfloat16*>(q_all);
   p.k_new = static_cast<const __nv_bfloat16*>(k_all);
   const bool tc_ok = choice != HEATKV_KERNEL_GENERIC && calib_tc_supported(ctx->calib_tc, p, ctx->cfg.d, n_seq);
-  for (int k = step_begin; k < step_end; ++k) {
+  // the small steps share one launch of the generic kernel (their query tiles side by side), longest first
+  AttnParams g = p;
+  g.cal_n = 0;
+  for (int k = step_end - 1; k >= step_begin; --k) {
     const bool use_tc = tc_ok && !(choice == HEATKV_KERNEL_AUTO && ctx->cfg.t[k] < 256);
     if (use_tc) {
       big[n_big] = k; big_t[n_big] = ctx->cfg.t[k]; big_tok0[n_big] = ctx->c[k] - ctx->cfg.t[k];
       ++n_big;
       continue;
     }
-    AttnParams g = p;                                   // a small step: the generic kernel on the step's views
-    g.q = p.q + (int64_t)(ctx->c[k] - ctx->cfg.t[k]) * s.q_tok;
-    g.seg_bias = seg_bias ? seg_bias + (int64_t)k * H * K : nullptr;
-    g.t_q = ctx->cfg.t[k];
-    g.n_own = ctx->c[k];
-    g.step = k;
-    g.beta_row = beta_layer + (int64_t)k * K;
+    g.cal_step[g.cal_n] = k;
+    g.cal_tile_begin[g.cal_n + 1] = g.cal_tile_begin[g.cal_n] + (ctx->cfg.t[k] + 63) / 64;
+    ++g.cal_n;
+  }
+  if (g.cal_n > 0) {
+    g.seg_bias = seg_bias;
+    g.cal_bias_stride = H * K;
+    g.beta_row = beta_layer;
     if (launch_attn_generic(g, ctx->cfg.d, n_seq, true, stream) != cudaSuccess) return HEATKV_ERR_CUDA;
     ctx->launches += 1;
     ctx->kstats.calibration_generic += 1;

@@ -76,8 +76,24 @@ __global__ void __launch_bounds__(GTHREADS, 2) attn_generic_kernel(const __grid_
     return;
   }
   const int seq = CALIB ? blockIdx.z : blockIdx.y;
-  const int q0 = blockIdx.x * GM;
   int head = CALIB ? blockIdx.y : blockIdx.z;
+  // What a CTA works on comes from the launch parameters; a calibration launch may cover several steps
+  // (heatkv_calibrate_scores_steps), its query tiles laid side by side along grid.x.
+  int t_q = p.t_q, n_own = p.n_own, step = p.step, q0 = blockIdx.x * GM;
+  const __nv_bfloat16* q_base = p.q;
+  float* beta_row = p.beta_row;
+  const float* seg_bias = p.seg_bias;
+  if (CALIB && p.cal_n > 0) {
+    int e = 0;
+    while (e + 1 < p.cal_n && (int)blockIdx.x >= p.cal_tile_begin[e + 1]) ++e;
+    step = p.cal_step[e];
+    n_own = p.c[step];
+    t_q = n_own - (step > 0 ? p.c[step - 1] : 0);
+    q0 = ((int)blockIdx.x - p.cal_tile_begin[e]) * GM;
+    q_base = p.q + (int64_t)(n_own - t_q) * p.q_tok;        // the step's queries on the token axis of all scales
+    beta_row = p.beta_row + (int64_t)step * p.K;              // p.beta_row is beta_accum[layer][0][0] here
+    if (seg_bias) seg_bias += (int64_t)step * p.cal_bias_stride;
+  }
 
   const int2* descs = nullptr;
   int n_desc = 0;
@@ -98,7 +114,7 @@ __global__ void __launch_bounds__(GTHREADS, 2) attn_generic_kernel(const __grid_
     }
     base_row = p.seqs[seq].base_row;
   }
-  const int n_own_tiles = (p.n_own + GN - 1) / GN;
+  const int n_own_tiles = (n_own + GN - 1) / GN;
   const int n_tiles = n_desc + n_own_tiles;
 
   const uint32_t sbase = smem_u32(smem);
@@ -126,7 +142,7 @@ __global__ void __launch_bounds__(GTHREADS, 2) attn_generic_kernel(const __grid_
       ks = kown + (int64_t)jj * GN * p.kv_tok;
       vs = vown ? vown + (int64_t)jj * GN * p.kv_tok : nullptr;
       stride = p.kv_tok;
-      nv = min(GN, p.n_own - jj * GN);
+      nv = min(GN, n_own - jj * GN);
     }
     load_tile<D>(sbase + SM::K_OFF + stage * SM::TILE_BYTES, ks, stride, nv, tid);
     if (vs) load_tile<D>(sbase + SM::V_OFF + stage * SM::TILE_BYTES, vs, stride, nv, tid);
@@ -135,8 +151,8 @@ __global__ void __launch_bounds__(GTHREADS, 2) attn_generic_kernel(const __grid_
 
   // ---- prologue: Q tile and the first GSTAGES - 1 key tiles, one copy group each (empty groups keep the count)
   {
-    const __nv_bfloat16* qsrc = p.q + seq * p.q_seq + head * p.q_head + (int64_t)q0 * p.q_tok;
-    load_tile<D>(sbase + SM::Q_OFF, qsrc, p.q_tok, min(GM, p.t_q - q0), tid);
+    const __nv_bfloat16* qsrc = q_base + seq * p.q_seq + head * p.q_head + (int64_t)q0 * p.q_tok;
+    load_tile<D>(sbase + SM::Q_OFF, qsrc, p.q_tok, min(GM, t_q - q0), tid);
     cp_async_commit();
     for (int j = 0; j < GSTAGES - 1; ++j) {
       if (j < n_tiles) issue_tile(j, j);
@@ -181,9 +197,9 @@ __global__ void __launch_bounds__(GTHREADS, 2) attn_generic_kernel(const __grid_
       seg_lo = seg_hi = (dsc.y >> 8) & 0xff;
     } else {
       int jj = j - n_desc;
-      nv = min(GN, p.n_own - jj * GN);
+      nv = min(GN, n_own - jj * GN);
       col0 = jj * GN;
-      seg_lo = seg_hi = p.step;
+      seg_lo = seg_hi = step;
       if (CALIB) {
         seg_lo = 0;
         while (p.c[seg_lo] <= col0) ++seg_lo;
@@ -211,7 +227,7 @@ __global__ void __launch_bounds__(GTHREADS, 2) attn_generic_kernel(const __grid_
     }
 
     // ---- scale, bias, mask, online softmax
-    const float* bias_h = p.seg_bias ? p.seg_bias + head * p.K : nullptr;
+    const float* bias_h = seg_bias ? seg_bias + head * p.K : nullptr;
     const float LOG2E = 1.4426950408889634f;
     float tile_bias = bias_h ? bias_h[seg_lo] * LOG2E : 0.f;
     float mx[2] = {-INFINITY, -INFINITY};
@@ -325,14 +341,14 @@ __global__ void __launch_bounds__(GTHREADS, 2) attn_generic_kernel(const __grid_
 
   if (CALIB) {
     // beta[step][sg] += (1/t) * sum over rows of mass(row, sg) / l(row)     (Eq. 2)
-    float* beta = p.beta_row + (int64_t)head * p.K * p.K;
-    for (int sg = 0; sg <= p.step; ++sg) {
+    float* beta = beta_row + (int64_t)head * p.K * p.K;
+    for (int sg = 0; sg <= step; ++sg) {
       float acc = 0.f;
       if (qd == 0) {
 #pragma unroll
         for (int r = 0; r < 2; ++r) {
           int row = warp * 16 + g + r * 8;
-          if (q0 + row < p.t_q)
+          if (q0 + row < t_q)
             acc += seg_sum[row * HEATKV_MAX_K + sg] * exp2f(seg_ref[row * HEATKV_MAX_K + sg] - m_run[r]) * inv_l[r];
         }
       }
@@ -342,9 +358,9 @@ __global__ void __launch_bounds__(GTHREADS, 2) attn_generic_kernel(const __grid_
       if (PARTIALS) {
         // slot of (CTA, warp, source scale); reduce_partials_kernel adds them up in a fixed order
         const int64_t cta = blockIdx.x + (int64_t)gridDim.x * (blockIdx.y + (int64_t)gridDim.y * blockIdx.z);
-        if (lane == 0) p.partials[(cta * (GTHREADS / 32) + warp) * HEATKV_MAX_K + sg] = acc / (float)p.t_q;
+        if (lane == 0) p.partials[(cta * (GTHREADS / 32) + warp) * HEATKV_MAX_K + sg] = acc / (float)t_q;
       } else {
-        if (lane == 0) atomicAdd(beta + sg, acc / (float)p.t_q);
+        if (lane == 0) atomicAdd(beta + sg, acc / (float)t_q);
       }
     }
   }
@@ -365,7 +381,7 @@ __global__ void __launch_bounds__(GTHREADS, 2) attn_generic_kernel(const __grid_
     __nv_bfloat16* dst = p.out + seq * p.o_seq + head * p.o_head + (int64_t)q0 * p.o_tok;
     for (int i = tid; i < GM * CH; i += GTHREADS) {
       int r = i / CH, ch = i % CH;
-      if (q0 + r < p.t_q) {
+      if (q0 + r < t_q) {
         int4 v = *reinterpret_cast<const int4*>(smem + SM::Q_OFF + tile_off<D>(r, ch));
         *reinterpret_cast<int4*>(dst + (int64_t)r * p.o_tok + ch * 8) = v;
       }
@@ -405,7 +421,8 @@ static cudaError_t launch_one(const AttnParams& p, int n_seq, cudaStream_t strea
     if (e != cudaSuccess) return e;
     configured[dev].store(true, std::memory_order_release);
   }
-  dim3 grid((p.t_q + GM - 1) / GM + (CALIB ? 0 : p.append_tiles), CALIB ? p.H : n_seq, CALIB ? n_seq : p.H);
+  const int q_tiles = CALIB && p.cal_n > 0 ? p.cal_tile_begin[p.cal_n] : (p.t_q + GM - 1) / GM;
+  dim3 grid(q_tiles + (CALIB ? 0 : p.append_tiles), CALIB ? p.H : n_seq, CALIB ? n_seq : p.H);
   kern<<<grid, GTHREADS, bytes, stream>>>(p);
   return cudaGetLastError();
 }

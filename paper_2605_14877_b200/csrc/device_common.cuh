@@ -56,6 +56,13 @@ struct AttnParams {
   // prior keys (count, and word offset of the first in the plan blob)
   int16_t table_ndesc[64];
   int32_t table_desc_begin[64];
+  // generic kernel, calibration over several steps in one launch (cal_n > 0): the query tiles of step cal_step[e]
+  // are blocks cal_tile_begin[e] .. cal_tile_begin[e + 1] - 1 of grid.x; q holds the queries of all scales, beta_row
+  // is beta_accum[layer][0][0], seg_bias the bias of step 0 with cal_bias_stride floats between steps
+  int32_t cal_n;
+  int32_t cal_tile_begin[HEATKV_MAX_K + 1];
+  int32_t cal_step[HEATKV_MAX_K];
+  int64_t cal_bias_stride;
 };
 
 struct CopyParams {
