@@ -475,6 +475,38 @@ def run_fp8_cache_workload(args):
         res[name + "_ms_per_scale"] = [round(float(x), 4) for x in ms]
         res[name + "_sum_ms"] = round(float(ms.sum()), 4)
         res[name + "_launches_per_sweep"] = int((hk.heatkv_launch_count(ses.ctx) - n0) // (reps + 2))
+
+        # the same sweep as one CUDA graph (what a generation loop would replay): launch gaps mostly gone
+        def sweep_once():
+            ids = [hk.heatkv_seq_open(ses.ctx, sch) for _ in range(sh.n_seq)]
+            for step in range(sh.K):
+                ses.pre_step(ids, step)
+                hk.heatkv_attention_append(ses.ctx, ids, 0, step, qs[step], ks[step], vs[step], None, None, outs[step])
+            for i in ids:
+                hk.heatkv_seq_close(ses.ctx, i)
+        side = torch.cuda.Stream()
+        side.wait_stream(torch.cuda.current_stream())
+        with torch.cuda.stream(side):
+            sweep_once()
+        torch.cuda.current_stream().wait_stream(side)
+        torch.cuda.synchronize()
+        g = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(g):
+            sweep_once()
+        g.replay()
+        torch.cuda.synchronize()
+        gms = 0.0
+        for rep in range(reps):
+            flush.fill_(2)
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            e0.record()
+            g.replay()
+            e1.record()
+            torch.cuda.synchronize()
+            gms += e0.elapsed_time(e1) / reps
+        assert hk.heatkv_device_status(ses.ctx) == 0
+        res[name + "_graph_sweep_ms"] = round(gms, 4)
+        del g
         hk.heatkv_schedule_free(sch)
         ses.close()
     print(json.dumps(res), flush=True)

@@ -141,8 +141,8 @@ typedef struct {
  * from k_new / v_new unquantised, as always): before the attention kernel runs, the call expands the visible
  * head-scales of its (layer, step) into bf16 staging rows inside the arena (stage_bytes), and the attention
  * kernels read those; the update after the layer quantises the new rows on their way into the pool.  Inputs
- * must be finite.  Only the paged layout is supported; heatkv_attention_append issues its parts as separate
- * kernels in such a context.  A call whose sequences need more staging rows than stage_bytes holds returns
+ * must be finite.  Only the paged layout is supported; heatkv_attention_append runs the expansion as a kernel of its
+ * own, and the update inside the attention launch only on the generic kernel (small steps).  A call whose sequences need more staging rows than stage_bytes holds returns
  * HEATKV_ERR_OUT_OF_PAGES (rows needed per sequence: the largest number of visible 64-row half-tiles of any
  * (layer, step) of its schedule, times 64).
  *

@@ -690,9 +690,15 @@ static int attention_impl(heatkv_ctx* ctx, const int* seq_ids, int n_seq, int la
       ctx->launches += 1;
       ctx->kstats.other += 1;
     }
-    for (int i = 0; i < n_seq; ++i) p.seqs[i].base_row = cp.stage_base[i];
+    for (int i = 0; i < n_seq; ++i) {
+      p.pool_base[i] = (int32_t)p.seqs[i].base_row;         // where a cache update riding on the launch writes
+      p.seqs[i].base_row = cp.stage_base[i];
+    }
+    p.k8_pool = ctx->k8_pool; p.v8_pool = ctx->v8_pool; p.k_exp = ctx->k_exp; p.v_exp = ctx->v_exp;
   }
-  bool fuse = with_update && stores && ctx->cfg.layout == HEATKV_LAYOUT_PAGED && !ctx->fp8;
+  // fp8 cache: only the generic kernel carries the quantising update (the same branch in the tensor-memory kernel's
+  // spare warps measured 1.5 % on the bf16 path's largest launch and 8 % on its smallest)
+  bool fuse = with_update && stores && ctx->cfg.layout == HEATKV_LAYOUT_PAGED && !(ctx->fp8 && use_tc);
   if (fuse) {
     // The tensor-memory kernel copies the new rows with two spare warps per SM beside the attention work, so
     // the update rides along whatever its size.  The generic kernel carries it as extra CTAs of its own
@@ -705,6 +711,8 @@ static int attention_impl(heatkv_ctx* ctx, const int* seq_ids, int n_seq, int la
       for (int hd = 0; hd < pe.sched.H; ++hd) storing += cnt[hd] > 0;
     }
     fuse = storing * (uint64_t)ctx->cfg.t[step] * ctx->cfg.d * 8 <= limit;
+    // (fp8 cache: a step that does not ride along goes through heatkv_append_compact below, which takes the
+    // sequences' pool rows from the context, not from p)
   }
   if (fuse) p.append_tiles = (ctx->cfg.t[step] + HEATKV_PAGE_TOKENS - 1) / HEATKV_PAGE_TOKENS + 1;
   cudaError_t e;

@@ -70,9 +70,13 @@ __global__ void __launch_bounds__(GTHREADS, 2) attn_generic_kernel(const __grid_
     // cache update riding on this launch: one CTA per (destination half-tile, sequence, head)
     const int sq = blockIdx.y, hd = blockIdx.z, j = blockIdx.x - (p.t_q + GM - 1) / GM;
     const int64_t src = sq * p.kv_seq + hd * p.kv_head;
-    append_half_tile(p.seqs[sq].plan, p.seqs[sq].base_row, (p.step * p.L + p.layer) * p.H + hd, j, p.k_new + src,
-                     p.v_new + src, p.kv_tok, const_cast<__nv_bfloat16*>(p.k_pool), const_cast<__nv_bfloat16*>(p.v_pool),
-                     D, threadIdx.x, GTHREADS);
+    if (p.k8_pool)
+      append_half_tile_fp8(p.seqs[sq].plan, p.pool_base[sq], (p.step * p.L + p.layer) * p.H + hd, j, p.k_new + src,
+                           p.v_new + src, p.kv_tok, p.k8_pool, p.v8_pool, p.k_exp, p.v_exp, D, threadIdx.x, GTHREADS);
+    else
+      append_half_tile(p.seqs[sq].plan, p.seqs[sq].base_row, (p.step * p.L + p.layer) * p.H + hd, j, p.k_new + src,
+                       p.v_new + src, p.kv_tok, const_cast<__nv_bfloat16*>(p.k_pool), const_cast<__nv_bfloat16*>(p.v_pool),
+                       D, threadIdx.x, GTHREADS);
     return;
   }
   const int seq = CALIB ? blockIdx.z : blockIdx.y;

@@ -63,6 +63,13 @@ struct AttnParams {
   int32_t cal_tile_begin[HEATKV_MAX_K + 1];
   int32_t cal_step[HEATKV_MAX_K];
   int64_t cal_bias_stride;
+  // fp8 cache (k8_pool != null): seqs[i].base_row numbers the bf16 staging rows the attention reads; a cache update
+  // riding on the launch quantises the new rows into the code pools, where sequence i starts at pool_base[i]
+  uint8_t* k8_pool;
+  uint8_t* v8_pool;
+  int8_t* k_exp;
+  int8_t* v_exp;
+  int32_t pool_base[HEATKV_MAX_BATCH];
 };
 
 struct CopyParams {
