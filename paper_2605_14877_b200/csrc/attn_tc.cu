@@ -699,38 +699,66 @@ attn_tc_kernel(const __grid_constant__ AttnParams p, const __grid_constant__ Map
             float* slots = p.split_partials + ((int64_t)seq * p.slots_per_seq + im.slot_base) * SPLIT_SLOT_FLOATS;
             float* slot_own = slots + (int64_t)im.sub * SPLIT_SLOT_FLOATS;
             int4* ocol = reinterpret_cast<int4*>(slot_own) + x * BM + row;
-#pragma unroll 1
-            for (int c = 0; c < D / 32; ++c) {
-              uint32_t r[32];
-              tmem_ld32(t_o + c * 32, r);
-              tmem_wait_ld();
-#pragma unroll
-              for (int gq = 0; gq < 8; ++gq)
-                ocol[(c * 8 + gq) * (2 * BM)] = make_int4((int)r[4 * gq], (int)r[4 * gq + 1], (int)r[4 * gq + 2], (int)r[4 * gq + 3]);
-            }
-            slot_own[2 * BM * D + x * BM + row] = m_ref;
-            slot_own[2 * BM * D + 2 * BM + x * BM + row] = l_sum;
-            __threadfence();
-            __syncwarp();
+            uint32_t* ctr = p.split_counters + ((int64_t)seq * p.ctrs_per_seq + im.ctr_base + qp) * 8 + (warp - 4);
+            // Every other piece of these 32 rows published already?  Then this warp's own stays in TMEM and it merges at once.
             uint32_t last = 0;
             if (lane == 0) {
-              uint32_t* ctr = p.split_counters + ((int64_t)seq * p.ctrs_per_seq + im.ctr_base + qp) * 8 + (warp - 4);
-              const uint32_t old = atomicAdd(ctr, 1u);
-              last = old == (uint32_t)(n_split - 1);
+              uint32_t seen;
+              asm volatile("ld.acquire.gpu.global.u32 %0, [%1];" : "=r"(seen) : "l"(ctr) : "memory");
+              last = seen == (uint32_t)(n_split - 1);
               if (last) *reinterpret_cast<volatile uint32_t*>(ctr) = 0;     // ready for the next launch
             }
             last = __shfl_sync(0xffffffffu, last, 0);
+            if (!last) {
+#pragma unroll 1
+              for (int c = 0; c < D / 32; ++c) {
+                uint32_t r[32];
+                tmem_ld32(t_o + c * 32, r);
+                tmem_wait_ld();
+#pragma unroll
+                for (int gq = 0; gq < 8; ++gq)
+                  ocol[(c * 8 + gq) * (2 * BM)] = make_int4((int)r[4 * gq], (int)r[4 * gq + 1], (int)r[4 * gq + 2], (int)r[4 * gq + 3]);
+              }
+              slot_own[2 * BM * D + x * BM + row] = m_ref;
+              slot_own[2 * BM * D + 2 * BM + x * BM + row] = l_sum;
+              __threadfence();
+              __syncwarp();
+              if (lane == 0) {
+                const uint32_t old = atomicAdd(ctr, 1u);
+                last = old == (uint32_t)(n_split - 1);
+                if (last) *reinterpret_cast<volatile uint32_t*>(ctr) = 0;   // ready for the next launch
+              }
+              last = __shfl_sync(0xffffffffu, last, 0);
+            }
             if (last) {
               __threadfence();
               // The pieces are added in piece order, this warp's own (still in TMEM) at its place among them, so
               // the result does not depend on which piece happened to arrive last.
+              // references and row sums of up to MERGE_FAST pieces are read once, all loads in flight together;
+              // a head cut finer than that reads them again where it needs them
+              constexpr int MERGE_FAST = 4;
+              float mp[MERGE_FAST], lp[MERGE_FAST];
+#pragma unroll
+              for (int s2 = 0; s2 < MERGE_FAST; ++s2) {
+                const float* sl = slots + (int64_t)(s2 * n_qp + qp) * SPLIT_SLOT_FLOATS;
+                const bool other = s2 < n_split && s2 != piece;
+                mp[s2] = other ? __ldcg(sl + 2 * BM * D + x * BM + row) : (s2 == piece ? m_ref : -INFINITY);
+                lp[s2] = other ? __ldcg(sl + 2 * BM * D + 2 * BM + x * BM + row) : (s2 == piece ? l_sum : 0.f);
+              }
               float m_all = -INFINITY;                                // common reference and total row sum
-              for (int s2 = 0; s2 < n_split; ++s2) {
+#pragma unroll
+              for (int s2 = 0; s2 < MERGE_FAST; ++s2) m_all = fmaxf(m_all, mp[s2]);
+              for (int s2 = MERGE_FAST; s2 < n_split; ++s2) {
                 const float* sl = slots + (int64_t)(s2 * n_qp + qp) * SPLIT_SLOT_FLOATS;
                 m_all = fmaxf(m_all, s2 == piece ? m_ref : __ldcg(sl + 2 * BM * D + x * BM + row));
               }
               float l_all = 0.f;
-              for (int s2 = 0; s2 < n_split; ++s2) {
+#pragma unroll
+              for (int s2 = 0; s2 < MERGE_FAST; ++s2) {               // piece order, as below
+                mp[s2] = s2 < n_split ? exp2f(mp[s2] - m_all) : 0.f;  // from here on: the piece's weight
+                l_all = fmaf(lp[s2], mp[s2], l_all);
+              }
+              for (int s2 = MERGE_FAST; s2 < n_split; ++s2) {
                 const float* sl = slots + (int64_t)(s2 * n_qp + qp) * SPLIT_SLOT_FLOATS;
                 const float l2 = s2 == piece ? l_sum : __ldcg(sl + 2 * BM * D + 2 * BM + x * BM + row);
                 const float m2 = s2 == piece ? m_ref : __ldcg(sl + 2 * BM * D + x * BM + row);
@@ -753,7 +781,12 @@ attn_tc_kernel(const __grid_constant__ AttnParams p, const __grid_constant__ Map
                     continue;
                   }
                   const float* sl = slots + (int64_t)(s2 * n_qp + qp) * SPLIT_SLOT_FLOATS;
-                  const float w = exp2f(__ldcg(sl + 2 * BM * D + x * BM + row) - m_all);
+                  float w;
+                  if (s2 < MERGE_FAST) {
+                    w = s2 == 0 ? mp[0] : s2 == 1 ? mp[1] : s2 == 2 ? mp[2] : mp[3];
+                  } else {
+                    w = exp2f(__ldcg(sl + 2 * BM * D + x * BM + row) - m_all);
+                  }
                   const float4* oc = reinterpret_cast<const float4*>(sl) + (c * 8) * (2 * BM) + x * BM + row;
 #pragma unroll
                   for (int i = 0; i < 8; ++i) {
