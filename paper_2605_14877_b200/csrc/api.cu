@@ -957,6 +957,19 @@ int heatkv_finalize_scores(heatkv_ctx* ctx, const float* beta_accum, int n_sampl
   return HEATKV_OK;
 }
 
+// Does the plan move any row at `step` in layers [l0, l1)?  phase 0: the eviction before the step (E_step),
+// phase 1: the eviction after a layer (G_step minus A_step of that layer).  The ragged layout launches its compaction
+// kernel only then.
+static bool plan_moves_rows(const Plan& pl, int phase, int step, int l0, int l1) {
+  const PlanHeader& hd = pl.header();
+  if (hd.n_move <= 0) return false;
+  const int32_t* cnt = pl.blob.data() + (phase == 0 ? hd.off_pre_cnt : hd.off_post_cnt);
+  for (int l = l0; l < l1; ++l)
+    for (int h = 0; h < hd.H; ++h)
+      if (cnt[((size_t)step * hd.L + l) * hd.H + h] > 0) return true;
+  return false;
+}
+
 int heatkv_append_compact(heatkv_ctx* ctx, const int* seq_ids, int n_seq, int layer, int step, const void* k_new,
                           const void* v_new, const heatkv_strides* st, void* stream_) {
   if (!ctx || !seq_ids || n_seq < 1 || n_seq > HEATKV_MAX_BATCH) return HEATKV_ERR_INVALID_ARG;
@@ -984,7 +997,7 @@ int heatkv_append_compact(heatkv_ctx* ctx, const int* seq_ids, int n_seq, int la
       const PlanEntry& pe = *ctx->plans[q->plan];
       p.seqs[i].plan = reinterpret_cast<const int32_t*>(ctx->meta + pe.meta_off);
       p.seqs[i].base_row = (int64_t)q->base_row;
-      moves |= pe.plan.header().n_move > 0;
+      moves |= plan_moves_rows(pe.plan, 0, step, l0, l1);
     }
     if (ctx->cfg.layout == HEATKV_LAYOUT_RAGGED && moves && step > 0) {
       p.phase = 0; p.layer_begin = l0; p.n_layers = l1 - l0; p.layer = l0;
@@ -1011,7 +1024,7 @@ int heatkv_append_compact(heatkv_ctx* ctx, const int* seq_ids, int n_seq, int la
   if (step + 1 < ctx->cfg.K) {                  // the last scale is never cached
     if (ctx->cfg.layout == HEATKV_LAYOUT_RAGGED) {
       bool moves = false;
-      for (int i = 0; i < n_seq; ++i) moves |= ctx->plans[ctx->seqs[seq_ids[i]].plan]->plan.header().n_move > 0;
+      for (int i = 0; i < n_seq; ++i) moves |= plan_moves_rows(ctx->plans[ctx->seqs[seq_ids[i]].plan]->plan, 1, step, layer, layer + 1);
       if (moves) {
         p.phase = 1; p.layer_begin = layer; p.n_layers = 1;
         if (launch_compact(p, n_seq, stream) != cudaSuccess) return HEATKV_ERR_CUDA;
