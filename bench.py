@@ -790,7 +790,7 @@ def main():
     flops = attention_flops(shape, am, n_seq)
     by = attention_bytes(shape, am, n_seq)
     calib_flops = sum(2 * shape.d * shape.t[k] * shape.c[k] for k in range(shape.K)) * shape.H * n_seq * len(CALIB_SEEDS)
-    tc_steps = [kk for kk in range(shape.K) if args.kernel != "generic" and (shape.t[kk] >= 256 or args.kernel == "tcgen05")]
+    tc_steps = [kk for kk in range(shape.K) if args.kernel != "generic" and (shape.t[kk] >= 256 or (shape.t[kk] >= 128 and n_seq * shape.H >= 64) or args.kernel == "tcgen05")]
 
     # ---- device-resident inputs of the timed workload: per layer, one [n_seq, H, t_k, d] block per scale
     # (N_LAYERS x 345 MB: every layer reads activations of its own, far more than the L2 holds)

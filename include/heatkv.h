@@ -70,7 +70,8 @@ typedef enum {
 } heatkv_accounting;
 
 typedef enum {
-  HEATKV_KERNEL_AUTO = 0,      /* tensor-memory kernel for large steps, generic otherwise */
+  HEATKV_KERNEL_AUTO = 0,      /* tensor-memory kernel for steps of >= 256 queries (>= 128 once a call holds
+                                  64 (sequence, head) units), generic otherwise */
   HEATKV_KERNEL_GENERIC = 1,   /* warp-level MMA kernel for every step                    */
   HEATKV_KERNEL_TCGEN05 = 2    /* tcgen05 / TMEM / TMA kernel wherever its shape rules allow */
 } heatkv_kernel_choice;

@@ -660,7 +660,9 @@ static int attention_impl(heatkv_ctx* ctx, const int* seq_ids, int n_seq, int la
   const bool stores = step + 1 < ctx->cfg.K;                  // the last scale is never cached
   const int choice = ctx->cfg.kernel;
   bool use_tc = choice != HEATKV_KERNEL_GENERIC && tc_supported(ctx->tc, p, ctx->cfg.d, n_seq, false);
-  if (choice == HEATKV_KERNEL_AUTO && p.t_q < 256) use_tc = false;
+  // AUTO: steps of 256 queries and more, and steps of 128 and more once the call holds 64 (sequence, head) units:
+  // from there on the warp-level kernel is bound by its mma.sync rate (144 queries, 128 units: 52 us against 23 us)
+  if (choice == HEATKV_KERNEL_AUTO && !(p.t_q >= 256 || (p.t_q >= 128 && (int64_t)n_seq * ctx->cfg.H >= 64))) use_tc = false;
   if (choice == HEATKV_KERNEL_TCGEN05 && !use_tc) return HEATKV_ERR_INVALID_ARG;   // never a silent substitute
   if (ctx->fp8) {
     // The attention kernels read bf16 rows: expand the visible head-scales of this (layer, step) from the code

@@ -120,10 +120,11 @@ def _run_full_parity(hk, sh, ref, make_schedule, layout, seed=0, bias=None, kern
         ks = hk.heatkv_kernel_launches(ses.ctx)
         if kernel == hk.KERNEL_TCGEN05:                     # forced: the tensor-memory kernel took every attention launch
             assert ks.tcgen05_attention_ready == 1 and ks.attention_generic == 0 and ks.attention_tcgen05 >= sh.K * sh.L
-        if kernel == hk.KERNEL_AUTO:                        # steps of 256 tokens and more go to the tensor-memory kernel
-            assert ks.tcgen05_attention_ready == 1
-            assert ks.attention_tcgen05 == sh.L * sum(1 for t in sh.t if t >= 256)
-            assert ks.attention_generic == sh.L * sum(1 for t in sh.t if t < 256)
+        if kernel == hk.KERNEL_AUTO:                        # steps of 256 tokens and more go to the tensor-memory kernel,
+            assert ks.tcgen05_attention_ready == 1          # steps of 128 and more once the call holds 64 (sequence, head) units
+            big = [t >= 256 or (t >= 128 and n_seq * sh.H >= 64) for t in sh.t]
+            assert ks.attention_tcgen05 == sh.L * sum(big)
+            assert ks.attention_generic == sh.L * (len(big) - sum(big))
         if want_kernels is not None:
             assert (ks.attention_tcgen05, ks.attention_generic) == want_kernels
         hk.heatkv_schedule_free(sch)
